@@ -1,0 +1,966 @@
+// Host side of the verification-step library: handle, workspace layout, kernel sequencing, CUDA-graph
+// replay of the decode loop, and the extern "C" entry points declared in include/aggressive_decoding.h.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <map>
+#include <string>
+#include <vector>
+
+#include "ad_common.cuh"
+#include "attention.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "steps.cuh"
+
+using namespace ad;
+
+namespace {
+
+enum PassKind { PK_VERIFY = 0, PK_DRAFT = 1, PK_ENCODE = 2, PK_COUNT = 3 };
+
+struct Mat {
+  const void* ptr = nullptr;
+  int N = 0, K = 0;
+  CUtensorMap map;
+};
+struct ActBuf {
+  void* ptr = nullptr;
+  int cols = 0;
+  CUtensorMap map[PK_COUNT];
+};
+struct EncLayer {
+  Mat wqkv, wo, w1, w2;
+  const float *bqkv, *bo, *ln1g, *ln1b, *b1, *b2, *ln2g, *ln2b;
+};
+struct DecLayer {
+  Mat wqkv, wo, cq, ckv, co, w1, w2;
+  const float *bqkv, *bo, *ln1g, *ln1b, *cbq, *cbkv, *cbo, *ln2g, *ln2b, *b1, *b2, *ln3g, *ln3b;
+};
+struct Model {
+  bool present = false;
+  Mat emb;
+  std::vector<EncLayer> enc;
+  std::vector<DecLayer> dec;
+  void* kenc = nullptr;   // [n_dec][B * max_src][d] cross-attention keys
+  void* venc = nullptr;
+};
+struct PassCfg {
+  int M_cap = 0;     // packed-token capacity of this pass kind
+  int ntile = 16;    // tokens per GEMM tile
+  int seg_max = 0;   // longest segment of one row
+  PassPlan plan;
+};
+
+thread_local std::string g_create_error;
+
+}  // namespace
+
+struct ad_handle {
+  ad_model_cfg cfg;
+  cudaStream_t stream = nullptr;
+  bool bf16 = false;
+  size_t esz = 4;            // bytes per activation / weight element
+  Model ar, nar;
+  PassCfg pass[PK_COUNT];
+  int M_all = 0;
+  Dims dims;
+  DevState st;
+  // activations
+  float *y = nullptr, *pre = nullptr;
+  ActBuf yb, abuf, hbuf, xg;
+  void *qbuf = nullptr, *ktmp = nullptr, *vtmp = nullptr, *kself = nullptr, *vself = nullptr, *encmem = nullptr;
+  float* part_val = nullptr;
+  int* part_idx = nullptr;
+  int n_vtiles = 0;
+  float* pe = nullptr;
+  int max_pos = 0;
+  int* ovr = nullptr;        // [B, max_tgt] staged draft-override stream
+  int* host_flag = nullptr;  // pinned
+  // state
+  int B = 0;                 // batch of the last ad_encode
+  bool encoded = false;
+  int last_vocab_which = -1;
+  std::string err;
+  struct GraphEntry { cudaGraphExec_t exec; int launches; };
+  std::map<std::string, GraphEntry> graphs;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
+  int launches = 0;          // kernels launched by the last ad_generate (direct) or per graph replay
+};
+
+namespace {
+
+#define AD_CUDA(h, call)                                                                      \
+  do {                                                                                        \
+    cudaError_t e__ = (call);                                                                 \
+    if (e__ != cudaSuccess) {                                                                 \
+      (h)->err = std::string(#call) + ": " + cudaGetErrorString(e__);                         \
+      return AD_ERR_CUDA;                                                                     \
+    }                                                                                         \
+  } while (0)
+
+int fail(ad_handle* h, int code, const std::string& msg) {
+  if (h) h->err = msg; else g_create_error = msg;
+  return code;
+}
+
+// ---- TMA descriptor encoding through the driver entry point (no link-time dependency on libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Row-major bf16 [rows, cols]; box = 64 columns (one 128-byte swizzle row) x box_rows.
+bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int pow2ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- workspace layout: one bump allocation pass, run with base = null to size it ----
+struct Bump {
+  char* base;
+  size_t off = 0;
+  explicit Bump(void* b) : base(static_cast<char*>(b)) {}
+  void* take(size_t bytes, size_t align = 1024) {
+    off = align_up(off, align);
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+void plan_take(Bump& bp, PassPlan& pl, int B, int M_cap) {
+  pl.M = (int*)bp.take(sizeof(int) * 4, 256);
+  pl.seg_off = (int*)bp.take(sizeof(int) * B, 256);
+  pl.seg_len = (int*)bp.take(sizeof(int) * B, 256);
+  pl.key_base = (int*)bp.take(sizeof(int) * B, 256);
+  pl.tok_row = (int*)bp.take(sizeof(int) * M_cap, 256);
+  pl.tok_pos = (int*)bp.take(sizeof(int) * M_cap, 256);
+  pl.tok_id = (int*)bp.take(sizeof(int) * M_cap, 256);
+  pl.kv_slot = (int*)bp.take(sizeof(int) * M_cap, 256);
+  pl.att_n = (int*)bp.take(sizeof(int) * M_cap, 256);
+}
+
+void pass_shapes(const ad_model_cfg& c, PassCfg* pass, int* M_all) {
+  const int B = c.max_batch;
+  pass[PK_VERIFY].seg_max = c.kmax;
+  pass[PK_DRAFT].seg_max = c.max_tgt + 1;
+  pass[PK_ENCODE].seg_max = c.max_src;
+  int all = 0;
+  for (int k = 0; k < PK_COUNT; ++k) {
+    pass[k].M_cap = B * pass[k].seg_max;
+    pass[k].ntile = clampi(pow2ceil(pass[k].M_cap), 16, 256);
+    if (pass[k].M_cap > all) all = pass[k].M_cap;
+  }
+  if (!c.has_drafter) { /* the drafter pass is never run; keep its shapes for sizing simplicity */ }
+  *M_all = all;
+}
+
+size_t layout(ad_handle* h, void* base) {
+  const ad_model_cfg& c = h->cfg;
+  const int B = c.max_batch, d = c.d_model, F = c.d_ffn;
+  const size_t e = h->esz;
+  Bump bp(base);
+  pass_shapes(c, h->pass, &h->M_all);
+  const int M_all = h->M_all, Mv = h->pass[PK_VERIFY].M_cap;
+  const int M_tmp = std::max(h->pass[PK_DRAFT].M_cap, h->pass[PK_ENCODE].M_cap);
+  h->y = (float*)bp.take(sizeof(float) * (size_t)M_all * d);
+  h->pre = (float*)bp.take(sizeof(float) * (size_t)M_all * d);
+  h->yb.ptr = bp.take(e * (size_t)M_all * d); h->yb.cols = d;
+  h->abuf.ptr = bp.take(e * (size_t)M_all * d); h->abuf.cols = d;
+  h->hbuf.ptr = bp.take(e * (size_t)M_all * F); h->hbuf.cols = F;
+  h->xg.ptr = bp.take(e * (size_t)M_all * d); h->xg.cols = d;
+  h->qbuf = bp.take(e * (size_t)M_all * d);
+  h->ktmp = bp.take(e * (size_t)M_tmp * d);
+  h->vtmp = bp.take(e * (size_t)M_tmp * d);
+  h->encmem = bp.take(e * (size_t)h->pass[PK_ENCODE].M_cap * d);
+  const size_t self_sz = e * (size_t)c.n_dec * B * c.max_tgt * d;
+  h->kself = bp.take(self_sz);
+  h->vself = bp.take(self_sz);
+  const size_t cross_sz = e * (size_t)c.n_dec * B * c.max_src * d;
+  h->ar.kenc = bp.take(cross_sz);
+  h->ar.venc = bp.take(cross_sz);
+  if (c.has_drafter) {
+    h->nar.kenc = bp.take(cross_sz);
+    h->nar.venc = bp.take(cross_sz);
+  }
+  h->n_vtiles = (c.vocab + 127) / 128;
+  h->part_val = (float*)bp.take(sizeof(float) * (size_t)h->n_vtiles * Mv);
+  h->part_idx = (int*)bp.take(sizeof(int) * (size_t)h->n_vtiles * Mv);
+  h->max_pos = std::max(c.max_src, c.max_tgt + 1);
+  h->pe = (float*)bp.take(sizeof(float) * (size_t)h->max_pos * d);
+  h->ovr = (int*)bp.take(sizeof(int) * (size_t)B * c.max_tgt);
+  for (int k = 0; k < PK_COUNT; ++k) plan_take(bp, h->pass[k].plan, B, h->pass[k].M_cap);
+  DevState& s = h->st;
+  auto ints = [&](size_t n) { return (int*)bp.take(sizeof(int) * n, 256); };
+  s.len = ints(B); s.last = ints(B); s.fin = ints(B); s.maxlen = ints(B); s.srclen = ints(B);
+  s.src = ints((size_t)B * c.max_src);
+  s.out_ids = ints((size_t)B * c.max_tgt);
+  s.drafts = ints((size_t)B * c.kmax); s.pred = ints((size_t)B * c.kmax); s.n_acc = ints(B);
+  s.stat_it = ints(B); s.stat_acc = ints(B); s.stat_off = ints(B);
+  s.loop_it = ints(4); s.status = ints(4); s.all_fin = ints(4);
+  s.cross_base = ints(B);
+  s.gidx = ints((size_t)B * c.kmax);
+  s.enc_slot = ints((size_t)B * c.max_src);
+  s.user_k = ints(B); s.user_n = ints(B); s.user_drafts = ints((size_t)B * c.kmax);
+  return align_up(bp.off, 1024);
+}
+
+int check_cfg(const ad_model_cfg* c, std::string* why) {
+  auto bad = [&](const char* m) { *why = m; return AD_ERR_ARG; };
+  if (!c) return bad("cfg is null");
+  if (c->d_model <= 0 || c->n_heads <= 0 || c->d_model % c->n_heads) return bad("d_model must be a positive multiple of n_heads");
+  const int dh = c->d_model / c->n_heads;
+  if (dh != 32 && dh != 64) return bad("head dimension must be 32 or 64");
+  if (c->d_ffn <= 0 || c->vocab <= 4 || c->n_enc < 1 || c->n_dec < 1) return bad("bad model sizes");
+  if (c->dtype != AD_DTYPE_FP32 && c->dtype != AD_DTYPE_BF16) return bad("dtype must be AD_DTYPE_FP32 or AD_DTYPE_BF16");
+  if (c->dtype == AD_DTYPE_BF16 && (c->d_model % 64 || c->d_ffn % 64)) return bad("BF16 needs d_model and d_ffn to be multiples of 64");
+  if (c->max_batch < 1 || c->max_batch > 256) return bad("max_batch must be 1..256");
+  if (c->max_src < 1 || c->max_tgt < 1) return bad("max_src and max_tgt must be positive");
+  if (c->kmax < 1 || c->kmax > 256 || c->kmax > c->max_tgt) return bad("kmax must be 1..min(256, max_tgt)");
+  const int ids[4] = {c->bos, c->pad, c->eos, c->mask};
+  for (int i = 0; i < 4; ++i) if (ids[i] < 0 || ids[i] >= c->vocab) return bad("special token id outside the vocabulary");
+  if (!(c->ln_eps >= 0.f)) return bad("ln_eps must be non-negative");
+  return AD_OK;
+}
+
+void weight_counts(const ad_model_cfg& c, size_t* mat, size_t* vec) {
+  const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+  *mat = V * d + (size_t)c.n_enc * (3 * d * d + d * d + 2 * d * F) + (size_t)c.n_dec * (3 * d * d + d * d + d * d + 2 * d * d + d * d + 2 * d * F);
+  *vec = (size_t)c.n_enc * (3 * d + d + 2 * d + F + d + 2 * d) + (size_t)c.n_dec * (3 * d + d + 2 * d + d + 2 * d + d + 2 * d + F + d + 2 * d);
+}
+
+int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
+  const ad_model_cfg& c = h->cfg;
+  const int d = c.d_model, F = c.d_ffn;
+  if (!w.matrices || !w.vectors) return fail(h, AD_ERR_ARG, "weight pointers are null");
+  if (reinterpret_cast<uintptr_t>(w.matrices) % 256) return fail(h, AD_ERR_ARG, "weight matrices must be 256-byte aligned");
+  const char* mp = static_cast<const char*>(w.matrices);
+  const float* vp = w.vectors;
+  bool ok = true;
+  auto mat = [&](Mat& t, int N, int K) {
+    t.ptr = mp; t.N = N; t.K = K;
+    mp += (size_t)N * K * h->esz;
+    if (h->bf16) ok = ok && make_map(&t.map, t.ptr, N, K, tc::BLOCK_N_FEAT);
+  };
+  auto vec = [&](const float*& t, int n) { t = vp; vp += n; };
+  mat(m.emb, c.vocab, d);
+  m.enc.resize(c.n_enc);
+  m.dec.resize(c.n_dec);
+  for (auto& L : m.enc) {
+    mat(L.wqkv, 3 * d, d); mat(L.wo, d, d); mat(L.w1, F, d); mat(L.w2, d, F);
+    vec(L.bqkv, 3 * d); vec(L.bo, d); vec(L.ln1g, d); vec(L.ln1b, d); vec(L.b1, F); vec(L.b2, d); vec(L.ln2g, d); vec(L.ln2b, d);
+  }
+  for (auto& L : m.dec) {
+    mat(L.wqkv, 3 * d, d); mat(L.wo, d, d); mat(L.cq, d, d); mat(L.ckv, 2 * d, d); mat(L.co, d, d); mat(L.w1, F, d); mat(L.w2, d, F);
+    vec(L.bqkv, 3 * d); vec(L.bo, d); vec(L.ln1g, d); vec(L.ln1b, d); vec(L.cbq, d); vec(L.cbkv, 2 * d); vec(L.cbo, d);
+    vec(L.ln2g, d); vec(L.ln2b, d); vec(L.b1, F); vec(L.b2, d); vec(L.ln3g, d); vec(L.ln3b, d);
+  }
+  if (!ok) return fail(h, AD_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+  m.present = true;
+  return AD_OK;
+}
+
+// ---- kernel launch helpers -----------------------------------------------------------------------
+
+int tc_stages(int ntile, int K) {
+  const int stage = tc::A_STAGE_BYTES + ntile * tc::BLOCK_K * 2;
+  int s = (200 * 1024) / stage;
+  s = clampi(s, 1, tc::MAX_STAGES);
+  const int kb = K / tc::BLOCK_K;
+  return s < kb ? s : (kb > 0 ? kb : 1);
+}
+
+template <int EPI>
+cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const GemmParams& p, int M_cap) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 204 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int stages = tc_stages(p.ntile, p.K);
+  const size_t smem = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2) + 1024;
+  dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile);
+  tc::gemm_tc_kernel<EPI><<<grid, 128, smem, st>>>(mw, mx, p, stages);
+  return cudaGetLastError();
+}
+
+template <int EPI>
+cudaError_t launch_simt(cudaStream_t st, const void* w, const void* x, const GemmParams& p, int M_cap) {
+  dim3 grid((p.N + 127) / 128, (M_cap + simt::TOK - 1) / simt::TOK);
+  simt::gemm_f32_kernel<EPI><<<grid, 128, 0, st>>>((const float*)w, (const float*)x, p);
+  return cudaGetLastError();
+}
+
+int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int* M_ptr, int M_cap, GemmParams p) {
+  p.K = W.K; p.N = W.N; p.M_ptr = M_ptr; p.M_cap = M_cap; p.status = h->st.status;
+  cudaError_t e;
+  h->launches++;
+  if (h->bf16) {
+    p.ntile = h->pass[pk].ntile;
+    switch (epi) {
+      case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, X.map[pk], p, M_cap); break;
+      case EPI_ACT: e = launch_tc<EPI_ACT>(h->stream, W.map, X.map[pk], p, M_cap); break;
+      case EPI_SCATTER: e = launch_tc<EPI_SCATTER>(h->stream, W.map, X.map[pk], p, M_cap); break;
+      default: e = launch_tc<EPI_ARGMAX>(h->stream, W.map, X.map[pk], p, M_cap); break;
+    }
+  } else {
+    p.ntile = simt::TOK;
+    switch (epi) {
+      case EPI_F32: e = launch_simt<EPI_F32>(h->stream, W.ptr, X.ptr, p, M_cap); break;
+      case EPI_ACT: e = launch_simt<EPI_ACT>(h->stream, W.ptr, X.ptr, p, M_cap); break;
+      case EPI_SCATTER: e = launch_simt<EPI_SCATTER>(h->stream, W.ptr, X.ptr, p, M_cap); break;
+      default: e = launch_simt<EPI_ARGMAX>(h->stream, W.ptr, X.ptr, p, M_cap); break;
+    }
+  }
+  if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("GEMM launch: ") + cudaGetErrorString(e));
+  return AD_OK;
+}
+
+int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, const void* v, void* out,
+              const int* key_base, const int* nkeys_tok, const int* nkeys_row) {
+  const ad_model_cfg& c = h->cfg;
+  AttnParams p;
+  p.q = q; p.k = k; p.v = v; p.out = out;
+  p.seg_off = pc.plan.seg_off; p.seg_len = pc.plan.seg_len;
+  p.key_base = key_base; p.nkeys_tok = nkeys_tok; p.nkeys_row = nkeys_row;
+  p.d = c.d_model;
+  p.qchunks = (pc.seg_max + ATT_QC - 1) / ATT_QC;
+  const int dh = c.d_model / c.n_heads;
+  p.scale = 1.0f / sqrtf((float)dh);
+  dim3 grid(h->dims.B * p.qchunks, c.n_heads);
+  h->launches++;
+  if (h->bf16) {
+    if (dh == 64) attention_kernel<bf16, 64><<<grid, 128, 0, h->stream>>>(p);
+    else attention_kernel<bf16, 32><<<grid, 128, 0, h->stream>>>(p);
+  } else {
+    if (dh == 64) attention_kernel<float, 64><<<grid, 128, 0, h->stream>>>(p);
+    else attention_kernel<float, 32><<<grid, 128, 0, h->stream>>>(p);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
+  return AD_OK;
+}
+
+int layernorm(ad_handle* h, const PassCfg& pc, const float* g, const float* b) {
+  const int d = h->cfg.d_model;
+  dim3 grid((pc.M_cap + 3) / 4);
+  h->launches++;
+  if (h->bf16) layernorm_kernel<bf16><<<grid, 128, 0, h->stream>>>(pc.plan.M, h->pre, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
+  else layernorm_kernel<float><<<grid, 128, 0, h->stream>>>(pc.plan.M, h->pre, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("layernorm launch: ") + cudaGetErrorString(e));
+  return AD_OK;
+}
+
+int embed(ad_handle* h, const PassCfg& pc, const Model& m) {
+  const int d = h->cfg.d_model;
+  const float sc = sqrtf((float)d);
+  h->launches++;
+  if (h->bf16) embed_kernel<bf16, bf16><<<pc.M_cap, 128, 0, h->stream>>>(pc.plan, (const bf16*)m.emb.ptr, h->pe, d, sc, h->y, (bf16*)h->yb.ptr);
+  else embed_kernel<float, float><<<pc.M_cap, 128, 0, h->stream>>>(pc.plan, (const float*)m.emb.ptr, h->pe, d, sc, h->y, (float*)h->yb.ptr);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("embed launch: ") + cudaGetErrorString(e));
+  return AD_OK;
+}
+
+#define AD_TRY(x) do { int rc__ = (x); if (rc__ != AD_OK) return rc__; } while (0)
+
+// Self-attention sublayer + FFN shared by the encoder and decoder layers.
+int self_attention_sublayer(ad_handle* h, int pk, const Mat& wqkv, const float* bqkv, const Mat& wo, const float* bo,
+                            const float* lng, const float* lnb, void* kbuf, void* vbuf) {
+  PassCfg& pc = h->pass[pk];
+  GemmParams p = {};
+  p.bias = bqkv; p.dst[0] = h->qbuf; p.dst[1] = kbuf; p.dst[2] = vbuf; p.seg_width = h->cfg.d_model; p.n_direct = 1;
+  p.slot = pc.plan.kv_slot;
+  AD_TRY(gemm(h, EPI_SCATTER, wqkv, h->yb, pk, pc.plan.M, pc.M_cap, p));
+  AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, nullptr));
+  GemmParams o = {};
+  o.bias = bo; o.out_f32 = h->pre; o.resid = h->y;
+  AD_TRY(gemm(h, EPI_F32, wo, h->abuf, pk, pc.plan.M, pc.M_cap, o));
+  return layernorm(h, pc, lng, lnb);
+}
+
+int ffn_sublayer(ad_handle* h, int pk, const Mat& w1, const float* b1, const Mat& w2, const float* b2, const float* lng,
+                 const float* lnb) {
+  PassCfg& pc = h->pass[pk];
+  GemmParams a = {};
+  a.bias = b1; a.relu = 1; a.out_act = h->hbuf.ptr;
+  AD_TRY(gemm(h, EPI_ACT, w1, h->yb, pk, pc.plan.M, pc.M_cap, a));
+  GemmParams o = {};
+  o.bias = b2; o.out_f32 = h->pre; o.resid = h->y;
+  AD_TRY(gemm(h, EPI_F32, w2, h->hbuf, pk, pc.plan.M, pc.M_cap, o));
+  return layernorm(h, pc, lng, lnb);
+}
+
+// Decoder stack over the packed tokens of pass pk (verification: cached, block-causal; drafter: no cache,
+// unmasked).  Leaves the final hidden states in yb.
+int decoder_pass(ad_handle* h, int pk, Model& m) {
+  const ad_model_cfg& c = h->cfg;
+  PassCfg& pc = h->pass[pk];
+  const size_t self_layer = (size_t)h->dims.max_tgt * c.max_batch * c.d_model * h->esz;
+  const size_t cross_layer = (size_t)c.max_src * c.max_batch * c.d_model * h->esz;
+  AD_TRY(embed(h, pc, m));
+  for (int l = 0; l < c.n_dec; ++l) {
+    DecLayer& L = m.dec[l];
+    void* kb = pk == PK_VERIFY ? (char*)h->kself + l * self_layer : h->ktmp;
+    void* vb = pk == PK_VERIFY ? (char*)h->vself + l * self_layer : h->vtmp;
+    AD_TRY(self_attention_sublayer(h, pk, L.wqkv, L.bqkv, L.wo, L.bo, L.ln1g, L.ln1b, kb, vb));
+    GemmParams q = {};
+    q.bias = L.cbq; q.out_act = h->qbuf;
+    AD_TRY(gemm(h, EPI_ACT, L.cq, h->yb, pk, pc.plan.M, pc.M_cap, q));
+    AD_TRY(attention(h, pc, h->qbuf, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
+                     h->st.cross_base, nullptr, h->st.srclen));
+    GemmParams o = {};
+    o.bias = L.cbo; o.out_f32 = h->pre; o.resid = h->y;
+    AD_TRY(gemm(h, EPI_F32, L.co, h->abuf, pk, pc.plan.M, pc.M_cap, o));
+    AD_TRY(layernorm(h, pc, L.ln2g, L.ln2b));
+    AD_TRY(ffn_sublayer(h, pk, L.w1, L.b1, L.w2, L.b2, L.ln3g, L.ln3b));
+  }
+  return AD_OK;
+}
+
+// Encoder stack + per-decoder-layer cross-attention key/value projection of the memory.
+int encoder_pass(ad_handle* h, Model& m, bool keep_memory) {
+  const ad_model_cfg& c = h->cfg;
+  PassCfg& pc = h->pass[PK_ENCODE];
+  const size_t cross_layer = (size_t)c.max_src * c.max_batch * c.d_model * h->esz;
+  AD_TRY(embed(h, pc, m));
+  for (int l = 0; l < c.n_enc; ++l) {
+    EncLayer& L = m.enc[l];
+    AD_TRY(self_attention_sublayer(h, PK_ENCODE, L.wqkv, L.bqkv, L.wo, L.bo, L.ln1g, L.ln1b, h->ktmp, h->vtmp));
+    AD_TRY(ffn_sublayer(h, PK_ENCODE, L.w1, L.b1, L.w2, L.b2, L.ln2g, L.ln2b));
+  }
+  if (keep_memory)
+    AD_CUDA(h, cudaMemcpyAsync(h->encmem, h->yb.ptr, (size_t)pc.M_cap * c.d_model * h->esz, cudaMemcpyDeviceToDevice, h->stream));
+  for (int l = 0; l < c.n_dec; ++l) {
+    DecLayer& L = m.dec[l];
+    GemmParams p = {};
+    p.bias = L.cbkv; p.dst[0] = (char*)m.kenc + l * cross_layer; p.dst[1] = (char*)m.venc + l * cross_layer;
+    p.seg_width = c.d_model; p.n_direct = 0; p.slot = h->st.enc_slot;
+    AD_TRY(gemm(h, EPI_SCATTER, L.ckv, h->yb, PK_ENCODE, pc.plan.M, pc.M_cap, p));
+  }
+  return AD_OK;
+}
+
+// Output projection fused with arg-max over X (yb for the verifier, the gathered mask rows for the drafter),
+// then the final reduction and (verifier) the draft compare.
+int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts) {
+  PassCfg& pc = h->pass[PK_VERIFY];
+  GemmParams p = {};
+  p.part_val = h->part_val; p.part_idx = h->part_idx;
+  AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
+  h->launches++;
+  argmax_accept_kernel<<<h->dims.B, 128, 0, h->stream>>>(h->st, pc.plan, h->dims, h->part_val, h->part_idx, h->n_vtiles,
+                                                       pc.M_cap, to_drafts);
+  AD_CUDA(h, cudaGetLastError());
+  h->last_vocab_which = to_drafts ? 1 : 0;
+  return AD_OK;
+}
+
+int prepare_verify(ad_handle* h, int source, int k_cap, const int* ovr, int ovr_len) {
+  h->launches++;
+  prepare_verify_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, source, k_cap, ovr,
+                                                 h->cfg.max_tgt, ovr_len);
+  AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+// Draft substep: sizes, drafter plan, drafter decoder, gather of the mask rows, projection + arg-max.
+int draft_stage(ad_handle* h, int k_cap) {
+  AD_TRY(prepare_verify(h, SRC_SIZES, k_cap, nullptr, 0));
+  h->launches++;
+  plan_draft_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->pass[PK_DRAFT].plan, h->dims);
+  AD_CUDA(h, cudaGetLastError());
+  AD_TRY(decoder_pass(h, PK_DRAFT, h->nar));
+  const int d = h->cfg.d_model;
+  PassCfg& pv = h->pass[PK_VERIFY];
+  h->launches++;
+  if (h->bf16) gather_rows_kernel<bf16><<<pv.M_cap, 128, 0, h->stream>>>(pv.plan.M, h->st.gidx, (const bf16*)h->yb.ptr, (bf16*)h->xg.ptr, d);
+  else gather_rows_kernel<float><<<pv.M_cap, 128, 0, h->stream>>>(pv.plan.M, h->st.gidx, (const float*)h->yb.ptr, (float*)h->xg.ptr, d);
+  AD_CUDA(h, cudaGetLastError());
+  return vocab_stage(h, h->nar, h->xg, 1);
+}
+
+int verify_stage(ad_handle* h) {
+  AD_TRY(decoder_pass(h, PK_VERIFY, h->ar));
+  return vocab_stage(h, h->ar, h->yb, 0);
+}
+
+int commit_stage(ad_handle* h, const int* n_dev) {
+  h->launches++;
+  commit_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, n_dev);
+  AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+// One iteration of the decode loop: draft -> verify -> commit, all on the device.
+int loop_iteration(ad_handle* h, const ad_gen_opts& o, const int* ovr, int ovr_len) {
+  if (o.mode == AD_MODE_GAD) {
+    if (o.run_drafter) {
+      AD_TRY(draft_stage(h, o.k));
+      AD_TRY(prepare_verify(h, SRC_KEEP, o.k, ovr, ovr_len));
+    } else {
+      AD_TRY(prepare_verify(h, SRC_OVERRIDE, o.k, ovr, ovr_len));
+    }
+  } else {
+    AD_TRY(prepare_verify(h, ovr ? SRC_OVERRIDE : SRC_POLICY, o.k, ovr, ovr_len));
+  }
+  AD_TRY(verify_stage(h));
+  return commit_stage(h, nullptr);
+}
+
+int read_status(ad_handle* h) {
+  int s = 0;
+  AD_CUDA(h, cudaMemcpyAsync(&s, h->st.status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  AD_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (s != 0) {
+    int z = 0;
+    cudaMemcpyAsync(h->st.status, &z, sizeof(int), cudaMemcpyHostToDevice, h->stream);
+    cudaStreamSynchronize(h->stream);
+    return fail(h, s, s == AD_ERR_TIMEOUT ? "a bounded device-side wait ran out" : "device-side argument check failed");
+  }
+  return AD_OK;
+}
+
+cudaMemcpyKind to_dev(int on_host) { return on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice; }
+cudaMemcpyKind from_dev(int on_host) { return on_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice; }
+
+void drop_graphs(ad_handle* h) {
+  for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second.exec);
+  h->graphs.clear();
+}
+
+}  // namespace
+
+// =====================================================================================================
+// extern "C"
+// =====================================================================================================
+
+extern "C" int ad_weight_counts(const ad_model_cfg* cfg, size_t* matrix_elems, size_t* vector_elems) {
+  std::string why;
+  if (check_cfg(cfg, &why) != AD_OK || !matrix_elems || !vector_elems) return fail(nullptr, AD_ERR_ARG, why.empty() ? "null output pointer" : why);
+  weight_counts(*cfg, matrix_elems, vector_elems);
+  return AD_OK;
+}
+
+extern "C" int ad_query_workspace(const ad_model_cfg* cfg, size_t* bytes) {
+  std::string why;
+  if (check_cfg(cfg, &why) != AD_OK || !bytes) return fail(nullptr, AD_ERR_ARG, why.empty() ? "null output pointer" : why);
+  ad_handle tmp;
+  tmp.cfg = *cfg;
+  tmp.bf16 = cfg->dtype == AD_DTYPE_BF16;
+  tmp.esz = tmp.bf16 ? 2 : 4;
+  *bytes = layout(&tmp, nullptr);
+  return AD_OK;
+}
+
+extern "C" const char* ad_last_error(const ad_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* workspace, size_t workspace_bytes,
+                         void* stream, ad_handle** out) {
+  std::string why;
+  if (!out) return fail(nullptr, AD_ERR_ARG, "out is null");
+  *out = nullptr;
+  if (check_cfg(cfg, &why) != AD_OK) return fail(nullptr, AD_ERR_ARG, why);
+  if (!w || !workspace) return fail(nullptr, AD_ERR_ARG, "weights or workspace is null");
+  if (reinterpret_cast<uintptr_t>(workspace) % 1024) return fail(nullptr, AD_ERR_ARG, "workspace must be 1024-byte aligned");
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return fail(nullptr, AD_ERR_CUDA, "no CUDA device");
+  if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
+
+  ad_handle* h = new ad_handle();
+  h->cfg = *cfg;
+  h->stream = static_cast<cudaStream_t>(stream);
+  h->bf16 = cfg->dtype == AD_DTYPE_BF16;
+  h->esz = h->bf16 ? 2 : 4;
+  const size_t need = layout(h, workspace);
+  auto bail = [&](int code, const std::string& msg) { g_create_error = msg; delete h; return code; };
+  if (need > workspace_bytes) return bail(AD_ERR_CAPACITY, "workspace too small: need " + std::to_string(need) + " bytes");
+  h->dims = Dims{cfg->max_batch, cfg->max_src, cfg->max_tgt, cfg->kmax, cfg->bos, cfg->pad, cfg->eos, cfg->mask};
+  int rc = bind_model(h, h->ar, w->ar);
+  if (rc == AD_OK && cfg->has_drafter) rc = bind_model(h, h->nar, w->nar);
+  if (rc != AD_OK) return bail(rc, h->err);
+  if (h->bf16) {
+    bool ok = true;
+    ActBuf* bufs[4] = {&h->yb, &h->abuf, &h->hbuf, &h->xg};
+    for (ActBuf* b : bufs)
+      for (int k = 0; k < PK_COUNT; ++k) ok = ok && make_map(&b->map[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile);
+    if (!ok) return bail(AD_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  }
+  // Cache, scratch and state start from zero so that no stale bit pattern is ever read as a number.
+  if (cudaMemsetAsync(workspace, 0, need, h->stream) != cudaSuccess) return bail(AD_ERR_CUDA, "clearing the workspace failed");
+  // Sinusoidal positional table PE(p, 2i) = sin(p / 10000^(2i/d)), PE(p, 2i+1) = cos(.), evaluated in double.
+  {
+    const int d = cfg->d_model;
+    std::vector<float> pe((size_t)h->max_pos * d);
+    for (int p = 0; p < h->max_pos; ++p)
+      for (int i = 0; i < d; i += 2) {
+        const double freq = exp(-log(10000.0) * (double)i / (double)d);
+        pe[(size_t)p * d + i] = (float)sin(p * freq);
+        if (i + 1 < d) pe[(size_t)p * d + i + 1] = (float)cos(p * freq);
+      }
+    if (cudaMemcpyAsync(h->pe, pe.data(), pe.size() * sizeof(float), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess)
+      return bail(AD_ERR_CUDA, "uploading the positional table failed");
+  }
+  if (cudaMallocHost(&h->host_flag, 64) != cudaSuccess) return bail(AD_ERR_CUDA, "cudaMallocHost failed");
+  if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess || cudaEventCreate(&h->ev2) != cudaSuccess)
+    return bail(AD_ERR_CUDA, "cudaEventCreate failed");
+  *out = h;
+  return AD_OK;
+}
+
+extern "C" int ad_destroy(ad_handle* h) {
+  if (!h) return AD_ERR_ARG;
+  cudaStreamSynchronize(h->stream);
+  drop_graphs(h);
+  if (h->host_flag) cudaFreeHost(h->host_flag);
+  if (h->ev0) cudaEventDestroy(h->ev0);
+  if (h->ev1) cudaEventDestroy(h->ev1);
+  if (h->ev2) cudaEventDestroy(h->ev2);
+  delete h;
+  return AD_OK;
+}
+
+extern "C" int ad_sync(ad_handle* h) {
+  if (!h) return AD_ERR_ARG;
+  return read_status(h);
+}
+
+extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, const int32_t* src_len, int32_t B,
+                         int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  const ad_model_cfg& c = h->cfg;
+  if (!src || !src_len) return fail(h, AD_ERR_ARG, "src or src_len is null");
+  if (B < 1 || B > c.max_batch) return fail(h, AD_ERR_CAPACITY, "B outside 1..max_batch");
+  if (src_stride < 1) return fail(h, AD_ERR_ARG, "src_stride must be positive");
+  if (on_host)
+    for (int b = 0; b < B; ++b)
+      if (src_len[b] < 1 || src_len[b] > c.max_src || src_len[b] > src_stride)
+        return fail(h, src_len[b] > c.max_src ? AD_ERR_CAPACITY : AD_ERR_ARG, "src_len outside 1..min(max_src, src_stride)");
+  if (B != h->B) drop_graphs(h);
+  h->B = B;
+  h->dims.B = B;
+  h->encoded = false;
+  const int w = src_stride < c.max_src ? src_stride : c.max_src;
+  AD_CUDA(h, cudaMemcpy2DAsync(h->st.src, sizeof(int) * c.max_src, src, sizeof(int) * src_stride, sizeof(int) * w, B, to_dev(on_host), h->stream));
+  AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, src_len, sizeof(int) * B, to_dev(on_host), h->stream));
+  h->launches++;
+  plan_encode_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_ENCODE].plan, h->dims);
+  AD_CUDA(h, cudaGetLastError());
+  AD_TRY(encoder_pass(h, h->ar, true));
+  if (c.has_drafter) AD_TRY(encoder_pass(h, h->nar, false));
+  h->encoded = true;
+  h->last_vocab_which = -1;
+  if (on_host) return read_status(h);
+  return AD_OK;
+}
+
+extern "C" int ad_verify_block(ad_handle* h, const int32_t* drafts, const int32_t* k, int32_t* argmax,
+                               int32_t* n_accepted, int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_verify_block before ad_encode");
+  if (!drafts || !k) return fail(h, AD_ERR_ARG, "drafts or k is null");
+  const ad_model_cfg& c = h->cfg;
+  const int B = h->B;
+  if (on_host)
+    for (int b = 0; b < B; ++b)
+      if (k[b] < 0 || k[b] > c.kmax) return fail(h, AD_ERR_ARG, "k outside 0..kmax");
+  AD_CUDA(h, cudaMemcpyAsync(h->st.user_drafts, drafts, sizeof(int) * (size_t)B * c.kmax, to_dev(on_host), h->stream));
+  AD_CUDA(h, cudaMemcpyAsync(h->st.user_k, k, sizeof(int) * B, to_dev(on_host), h->stream));
+  AD_TRY(prepare_verify(h, SRC_USER, c.kmax, nullptr, 0));
+  AD_TRY(verify_stage(h));
+  if (on_host) {
+    if (argmax) AD_CUDA(h, cudaMemcpyAsync(argmax, h->st.pred, sizeof(int) * (size_t)B * c.kmax, cudaMemcpyDeviceToHost, h->stream));
+    if (n_accepted) AD_CUDA(h, cudaMemcpyAsync(n_accepted, h->st.n_acc, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
+    return read_status(h);
+  }
+  h->launches++;
+  export_block_kernel<<<B, 64, 0, h->stream>>>(h->st, h->dims, argmax, n_accepted, nullptr, nullptr, h->pass[PK_VERIFY].plan);
+  AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+extern "C" int ad_commit(ad_handle* h, const int32_t* n, int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_commit before ad_encode");
+  const int* n_dev = nullptr;
+  if (n) {
+    AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, n, sizeof(int) * h->B, to_dev(on_host), h->stream));
+    n_dev = h->st.user_n;
+  }
+  AD_TRY(commit_stage(h, n_dev));
+  if (on_host) return read_status(h);
+  return AD_OK;
+}
+
+extern "C" int ad_draft_block(ad_handle* h, int32_t k_cap, int32_t* drafts, int32_t* k, int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_draft_block before ad_encode");
+  if (!h->cfg.has_drafter) return fail(h, AD_ERR_STATE, "the handle has no drafter model");
+  const ad_model_cfg& c = h->cfg;
+  if (k_cap < 1 || k_cap > c.kmax) return fail(h, AD_ERR_ARG, "k_cap outside 1..kmax");
+  AD_TRY(draft_stage(h, k_cap));
+  const int B = h->B;
+  if (on_host) {
+    if (drafts) AD_CUDA(h, cudaMemcpyAsync(drafts, h->st.drafts, sizeof(int) * (size_t)B * c.kmax, cudaMemcpyDeviceToHost, h->stream));
+    if (k) AD_CUDA(h, cudaMemcpyAsync(k, h->pass[PK_VERIFY].plan.seg_len, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
+    return read_status(h);
+  }
+  h->launches++;
+  export_block_kernel<<<B, 64, 0, h->stream>>>(h->st, h->dims, nullptr, nullptr, drafts, k, h->pass[PK_VERIFY].plan);
+  AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+extern "C" int ad_get_state(ad_handle* h, int32_t* len, int32_t* last_tok, int32_t* finished) {
+  if (!h) return AD_ERR_ARG;
+  if (h->B < 1) return fail(h, AD_ERR_STATE, "ad_get_state before ad_encode");
+  if (len) AD_CUDA(h, cudaMemcpyAsync(len, h->st.len, sizeof(int) * h->B, cudaMemcpyDeviceToHost, h->stream));
+  if (last_tok) AD_CUDA(h, cudaMemcpyAsync(last_tok, h->st.last, sizeof(int) * h->B, cudaMemcpyDeviceToHost, h->stream));
+  if (finished) AD_CUDA(h, cudaMemcpyAsync(finished, h->st.fin, sizeof(int) * h->B, cudaMemcpyDeviceToHost, h->stream));
+  return read_status(h);
+}
+
+extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride, const int32_t* src_len, int32_t B,
+                           const ad_gen_opts* opts, int32_t* out, int32_t out_stride, int32_t* out_len,
+                           ad_stats* stats, int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  const ad_model_cfg& c = h->cfg;
+  if (!opts || !out || !out_len) return fail(h, AD_ERR_ARG, "opts, out or out_len is null");
+  if (opts->mode != AD_MODE_IAD && opts->mode != AD_MODE_GAD) return fail(h, AD_ERR_ARG, "unknown mode");
+  if (opts->k < 1 || opts->k > c.kmax) return fail(h, AD_ERR_ARG, "k outside 1..kmax");
+  if (opts->mode == AD_MODE_GAD && opts->run_drafter && !c.has_drafter) return fail(h, AD_ERR_STATE, "GAD with run_drafter needs a drafter model");
+  if (opts->mode == AD_MODE_GAD && !opts->run_drafter && !opts->draft_override) return fail(h, AD_ERR_ARG, "GAD without the drafter needs draft_override");
+  if (opts->draft_override && opts->override_stride < 1) return fail(h, AD_ERR_ARG, "override_stride must be positive");
+  if (out_stride < 1) return fail(h, AD_ERR_ARG, "out_stride must be positive");
+
+  AD_CUDA(h, cudaEventRecord(h->ev0, h->stream));
+  h->launches = 0;
+  AD_TRY(ad_encode(h, src, src_stride, src_len, B, on_host));
+  int max_iters = c.max_tgt;
+  if (opts->max_len) {
+    AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, opts->max_len, sizeof(int) * B, to_dev(on_host), h->stream));
+    h->launches++;
+    set_maxlen_kernel<<<(B + 63) / 64, 64, 0, h->stream>>>(h->st, h->dims, h->st.user_n);
+    AD_CUDA(h, cudaGetLastError());
+    if (on_host) {
+      max_iters = 1;
+      for (int b = 0; b < B; ++b) {
+        if (opts->max_len[b] < 1 || opts->max_len[b] > c.max_tgt) return fail(h, AD_ERR_ARG, "max_len outside 1..max_tgt");
+        if (opts->max_len[b] > max_iters) max_iters = opts->max_len[b];
+      }
+    }
+  }
+  const int* ovr = nullptr;
+  int ovr_len = 0;   // valid leading entries of each staged override row
+  if (opts->draft_override) {
+    ovr_len = opts->override_stride < c.max_tgt ? opts->override_stride : c.max_tgt;
+    AD_CUDA(h, cudaMemcpy2DAsync(h->ovr, sizeof(int) * c.max_tgt, opts->draft_override, sizeof(int) * opts->override_stride,
+                                 sizeof(int) * ovr_len, B, to_dev(on_host), h->stream));
+    ovr = h->ovr;
+  }
+  AD_CUDA(h, cudaEventRecord(h->ev1, h->stream));
+
+  cudaGraphExec_t exec = nullptr;
+  int per_iter_launches = 0;
+  if (opts->use_graph && h->stream != nullptr) {   // the legacy default stream cannot be captured
+    char key[160];
+    snprintf(key, sizeof(key), "B%d m%d k%d o%d v%d d%d", B, opts->mode, opts->k, ovr ? 1 : 0, ovr_len, opts->run_drafter);
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+      cudaGraph_t g = nullptr;
+      const int before = h->launches;
+      AD_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      const int rc = loop_iteration(h, *opts, ovr, ovr_len);
+      cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+      per_iter_launches = h->launches - before;
+      h->launches = before;
+      if (rc != AD_OK) { if (g) cudaGraphDestroy(g); return rc; }
+      if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+      e = cudaGraphInstantiate(&exec, g, 0);
+      cudaGraphDestroy(g);
+      if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+      h->graphs[key] = ad_handle::GraphEntry{exec, per_iter_launches};
+    } else {
+      exec = it->second.exec;
+      per_iter_launches = it->second.launches;
+    }
+  }
+
+  const int sync_every = opts->sync_every > 0 ? opts->sync_every : 4;
+  int iters = 0;
+  volatile int* flag = h->host_flag;
+  flag[0] = 0;
+  while (iters < max_iters + sync_every) {
+    for (int s = 0; s < sync_every; ++s, ++iters) {
+      if (exec) {
+        AD_CUDA(h, cudaGraphLaunch(exec, h->stream));
+        h->launches += per_iter_launches;
+      } else {
+        AD_TRY(loop_iteration(h, *opts, ovr, ovr_len));
+      }
+    }
+    AD_CUDA(h, cudaMemcpyAsync(h->host_flag, h->st.all_fin, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (flag[0]) break;
+  }
+  AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
+  const int w = out_stride < c.max_tgt ? out_stride : c.max_tgt;
+  AD_CUDA(h, cudaMemcpy2DAsync(out, sizeof(int) * out_stride, h->st.out_ids, sizeof(int) * c.max_tgt, sizeof(int) * w, B, from_dev(on_host), h->stream));
+  AD_CUDA(h, cudaMemcpyAsync(out_len, h->st.len, sizeof(int) * B, from_dev(on_host), h->stream));
+  if (stats) {
+    std::vector<int> buf(3 * (size_t)B + 1);
+    AD_CUDA(h, cudaMemcpyAsync(buf.data(), h->st.stat_it, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(buf.data() + B, h->st.stat_acc, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(buf.data() + 2 * B, h->st.stat_off, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(buf.data() + 3 * B, h->st.loop_it, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaStreamSynchronize(h->stream));
+    memset(stats, 0, sizeof(*stats));
+    for (int b = 0; b < B; ++b) {
+      stats->row_iterations += buf[b];
+      stats->accepted += buf[B + b];
+      stats->offered += buf[2 * B + b];
+    }
+    stats->iterations = buf[3 * B];
+    cudaEventElapsedTime(&stats->encode_ms, h->ev0, h->ev1);
+    cudaEventElapsedTime(&stats->device_ms, h->ev1, h->ev2);
+  }
+  return read_status(h);
+}
+
+extern "C" int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_elems) {
+  if (!h || !logits) return AD_ERR_ARG;
+  if (h->last_vocab_which != which) return fail(h, AD_ERR_STATE, "no matching projection has just run");
+  PassCfg& pc = h->pass[PK_VERIFY];
+  int M = 0;
+  AD_CUDA(h, cudaMemcpyAsync(&M, pc.plan.M, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  AD_CUDA(h, cudaStreamSynchronize(h->stream));
+  if ((size_t)M * h->cfg.vocab > capacity_elems) return fail(h, AD_ERR_CAPACITY, "logits buffer too small");
+  Model& m = which == 1 ? h->nar : h->ar;
+  GemmParams p = {};
+  p.out_f32 = logits;
+  AD_TRY(gemm(h, EPI_F32, m.emb, which == 1 ? h->xg : h->yb, PK_VERIFY, pc.plan.M, pc.M_cap, p));
+  return AD_OK;
+}
+
+extern "C" int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size_t capacity_elems) {
+  if (!h || !mem) return AD_ERR_ARG;
+  if (!h->encoded || b < 0 || b >= h->B) return fail(h, AD_ERR_STATE, "no encoded row b");
+  PassPlan& pl = h->pass[PK_ENCODE].plan;
+  int off = 0, len = 0;
+  AD_CUDA(h, cudaMemcpyAsync(&off, pl.seg_off + b, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  AD_CUDA(h, cudaMemcpyAsync(&len, pl.seg_len + b, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  AD_CUDA(h, cudaStreamSynchronize(h->stream));
+  const size_t n = (size_t)len * h->cfg.d_model;
+  if (n > capacity_elems) return fail(h, AD_ERR_CAPACITY, "memory buffer too small");
+  const size_t start = (size_t)off * h->cfg.d_model;
+  if (h->bf16) to_f32_kernel<bf16><<<64, 256, 0, h->stream>>>((const bf16*)h->encmem + start, mem, n);
+  else to_f32_kernel<float><<<64, 256, 0, h->stream>>>((const float*)h->encmem + start, mem, n);
+  AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+// ---- single-kernel entry points -----------------------------------------------------------------
+
+extern "C" size_t ad_vocab_argmax_scratch_bytes(int32_t vocab, int32_t M) {
+  const size_t tiles = (size_t)(vocab + 127) / 128;
+  return align_up(tiles * (size_t)M * sizeof(float), 256) + align_up(tiles * (size_t)M * sizeof(int), 256);
+}
+
+namespace {
+
+// Arg-max over tiles for M rows without any decoding state.  grid = M, block = 32.
+__global__ void argmax_rows_kernel(const float* __restrict__ part_val, const int* __restrict__ part_idx, int n_tiles,
+                                   int M_cap, int* __restrict__ out) {
+  const int m = blockIdx.x, lane = threadIdx.x;
+  float v = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int t = lane; t < n_tiles; t += 32) {
+    const float ov = part_val[(size_t)t * M_cap + m];
+    const int oi = part_idx[(size_t)t * M_cap + m];
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+  tc::warp_argmax(v, idx);
+  if (lane == 0) out[m] = idx;
+}
+
+}  // namespace
+
+extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d, int32_t vocab,
+                               int32_t* argmax, void* scratch, size_t scratch_bytes, int32_t* status, void* stream) {
+  if (!x || !emb || !argmax || !scratch || M < 1 || d < 1 || vocab < 1) return AD_ERR_ARG;
+  if (scratch_bytes < ad_vocab_argmax_scratch_bytes(vocab, M)) return AD_ERR_CAPACITY;
+  if (reinterpret_cast<uintptr_t>(scratch) % 256) return AD_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int tiles = (vocab + 127) / 128;
+  float* pv = static_cast<float*>(scratch);
+  int* pi = reinterpret_cast<int*>(static_cast<char*>(scratch) + align_up((size_t)tiles * M * sizeof(float), 256));
+  GemmParams p = {};
+  p.K = d; p.N = vocab; p.M_ptr = nullptr; p.M_host = M; p.M_cap = M; p.part_val = pv; p.part_idx = pi; p.status = status;
+  cudaError_t e;
+  if (dtype == AD_DTYPE_BF16) {
+    if (d % 64 || M > 256) return AD_ERR_ARG;
+    CUtensorMap mw, mx;
+    p.ntile = clampi(pow2ceil(M), 16, 256);
+    if (!make_map(&mw, emb, vocab, d, tc::BLOCK_N_FEAT) || !make_map(&mx, x, M, d, p.ntile)) return AD_ERR_CUDA;
+    e = launch_tc<EPI_ARGMAX>(st, mw, mx, p, M);
+  } else if (dtype == AD_DTYPE_FP32) {
+    p.ntile = simt::TOK;
+    e = launch_simt<EPI_ARGMAX>(st, emb, x, p, M);
+  } else {
+    return AD_ERR_ARG;
+  }
+  if (e != cudaSuccess) return AD_ERR_CUDA;
+  argmax_rows_kernel<<<M, 32, 0, st>>>(pv, pi, tiles, M, argmax);
+  return cudaGetLastError() == cudaSuccess ? AD_OK : AD_ERR_CUDA;
+}
+
+extern "C" int ad_linear(const void* x, const void* W, const float* bias, int32_t dtype, int32_t M, int32_t K,
+                         int32_t N, float* y, int32_t* status, void* stream) {
+  if (!x || !W || !y || M < 1 || K < 1 || N < 1) return AD_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  GemmParams p = {};
+  p.K = K; p.N = N; p.M_ptr = nullptr; p.M_host = M; p.M_cap = M; p.bias = bias; p.out_f32 = y; p.status = status;
+  cudaError_t e;
+  if (dtype == AD_DTYPE_BF16) {
+    if (K % 64 || M > 256) return AD_ERR_ARG;
+    CUtensorMap mw, mx;
+    p.ntile = clampi(pow2ceil(M), 16, 256);
+    if (!make_map(&mw, W, N, K, tc::BLOCK_N_FEAT) || !make_map(&mx, x, M, K, p.ntile)) return AD_ERR_CUDA;
+    e = launch_tc<EPI_F32>(st, mw, mx, p, M);
+  } else if (dtype == AD_DTYPE_FP32) {
+    p.ntile = simt::TOK;
+    e = launch_simt<EPI_F32>(st, W, x, p, M);
+  } else {
+    return AD_ERR_ARG;
+  }
+  return e == cudaSuccess ? AD_OK : AD_ERR_CUDA;
+}

@@ -1,0 +1,281 @@
+// BF16 projection GEMM on the 5th-generation tensor cores (tcgen05.mma, accumulator in tensor memory),
+// operands staged in shared memory by TMA through an mbarrier ring.
+//
+// Computes D^T[n, m] = sum_k W[n, k] * X[m, k]  ("swap-AB"): the 128 rows of a weight tile fill the MMA's
+// M side (one TMEM lane per output feature) and the packed tokens are the MMA's N side, so a block of a few
+// drafted tokens still issues full-width instructions and the kernel streams every weight byte exactly once.
+// Both operands are K-major (row-major [rows, K]) and land in shared memory in the 128-byte-swizzled
+// canonical layout that the TMA and the MMA shared-memory descriptor agree on.
+//
+// Thread roles inside the 128-thread CTA: lane 0 of warp 0 issues TMA loads, lane 0 of warp 1 issues the
+// MMAs, then all four warps read their 32 TMEM lanes back (tcgen05.ld 32x32b) for the epilogue.
+// Every mbarrier wait is bounded; on expiry the kernel latches AD_ERR_TIMEOUT, frees its TMEM and returns.
+#pragma once
+
+#include "ad_common.cuh"
+
+namespace ad {
+namespace tc {
+
+constexpr int BLOCK_N_FEAT = 128;   // weight rows per CTA = MMA M
+constexpr int BLOCK_K = 64;         // bf16 elements per 128-byte swizzle row
+constexpr int UMMA_K = 16;          // K of one tcgen05.mma kind::f16
+constexpr int A_STAGE_BYTES = BLOCK_N_FEAT * BLOCK_K * 2;   // 16 KiB
+constexpr int MAX_STAGES = 8;
+constexpr uint32_t SPIN_LIMIT = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (after latching the error) when the phase did not complete in time.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  for (uint32_t i = 0; i < SPIN_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  latch_error(status, AD_ERR_TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) and whose 8-row
+// groups are 1024 bytes apart, 128-byte swizzle: start address >> 4 in bits [0,14), leading byte offset
+// (unused by swizzled K-major layouts, encoded as 1) in [16,30), stride byte offset 1024 >> 4 in [32,46),
+// descriptor version 1 in [46,48), layout type 2 (SWIZZLE_128B) in [61,64).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr >> 4) & 0x3FFF);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+// Instruction descriptor of kind::f16 with BF16 A and B (both K-major), FP32 accumulator:
+// accumulator format 1 (F32) in bits [4,6), A format 1 (BF16) in [7,10), B format 1 in [10,13),
+// N >> 3 in [17,23), M >> 4 in [24,29).
+__device__ __forceinline__ uint32_t make_idesc(int mma_m, int mma_n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(mma_n >> 3) << 17) |
+         (static_cast<uint32_t>(mma_m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Makes the mbarrier track completion of every MMA this thread has issued so far.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Best (value, lowest index) over the 32 lanes of a warp.
+__device__ __forceinline__ void warp_argmax(float& v, int& i) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, v, off);
+    int oi = __shfl_xor_sync(0xffffffffu, i, off);
+    if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+  }
+}
+
+// Applies the epilogue to 16 consecutive tokens (m0 .. m0+15) of output feature n held by this thread.
+template <int EPI, typename ActT>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int n, int m0, int M, const float* acc) {
+  if (n >= p.N) return;
+  const float b = p.bias ? p.bias[n] : 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const int m = m0 + j;
+    if (m >= M) break;
+    float v = acc[j] + b;
+    if (EPI == EPI_F32) {
+      if (p.resid) v += p.resid[(size_t)m * p.N + n];
+      p.out_f32[(size_t)m * p.N + n] = v;
+    } else if (EPI == EPI_ACT) {
+      if (p.relu) v = fmaxf(v, 0.f);
+      reinterpret_cast<ActT*>(p.out_act)[(size_t)m * p.N + n] = from_f32<ActT>(v);
+    } else if (EPI == EPI_SCATTER) {
+      const int s = n / p.seg_width, c = n - s * p.seg_width;
+      const int row = (s < p.n_direct) ? m : p.slot[m];
+      reinterpret_cast<ActT*>(p.dst[s])[(size_t)row * p.seg_width + c] = from_f32<ActT>(v);
+    }
+  }
+}
+
+// grid = (ceil(N / 128), ceil(M_cap / ntile)); block = 128 threads; dynamic smem = stages * stage bytes + 1024.
+template <int EPI>
+__global__ void __launch_bounds__(128, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+               const GemmParams p, const int stages) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];
+  __shared__ __align__(8) uint64_t bar_empty[MAX_STAGES];
+  __shared__ __align__(8) uint64_t bar_acc;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ float red_val[4][256];
+  __shared__ int red_idx[4][256];
+
+  const int M = p.M_ptr ? *p.M_ptr : p.M_host;
+  const int t0 = blockIdx.y * p.ntile;
+  if (t0 >= M) return;                       // uniform over the CTA: nothing allocated yet
+  const int n0 = blockIdx.x * BLOCK_N_FEAT;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntile = p.ntile;
+  const int b_stage_bytes = ntile * BLOCK_K * 2;
+  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  const int num_kb = p.K / BLOCK_K;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < (uint32_t)ntile) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bar_acc), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // one full warp allocates the accumulator columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&tmem_base_slot)), "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = tmem_base_slot;
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer ----
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % stages;
+      const uint32_t round = kb / stages;
+      if (round > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (round - 1) & 1, p.status)) { abort_flag = 1; break; }
+      if (*reinterpret_cast<volatile int*>(&abort_flag)) break;
+      const uint32_t a_dst = smem_base + s * stage_bytes;
+      const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+      const uint32_t bar = smem_u32(&bar_full[s]);
+      mbar_expect_tx(bar, (uint32_t)stage_bytes);
+      tma_load_2d(a_dst, &map_w, kb * BLOCK_K, n0, bar);
+      tma_load_2d(b_dst, &map_x, kb * BLOCK_K, t0, bar);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer ----
+    const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % stages;
+      const uint32_t round = kb / stages;
+      ok = mbar_wait(smem_u32(&bar_full[s]), round & 1, p.status);
+      if (!ok) { abort_flag = 1; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a_addr = smem_base + s * stage_bytes;
+      const uint64_t desc_a = make_smem_desc(a_addr);
+      const uint64_t desc_b = make_smem_desc(a_addr + A_STAGE_BYTES);
+#pragma unroll
+      for (int k4 = 0; k4 < BLOCK_K / UMMA_K; ++k4) {
+        // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
+        umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+      }
+      umma_commit(smem_u32(&bar_empty[s]));   // stage reusable once these MMAs have read it
+    }
+    if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
+  }
+  __syncwarp();
+
+  // ---- epilogue: all four warps ----
+  bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.status);
+  if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
+  ready = __all_sync(0xffffffffu, ready);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (ready) {
+    const int n = n0 + warp * 32 + lane;
+    for (int c = 0; c < ntile; c += 16) {
+      float acc[16];
+      tmem_ld16(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c), acc);
+      if (EPI == EPI_ARGMAX) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float v = (n < p.N) ? acc[j] : -INFINITY;
+          int i = n;
+          warp_argmax(v, i);
+          if (lane == 0) { red_val[warp][c + j] = v; red_idx[warp][c + j] = i; }
+        }
+      } else {
+        epilogue_chunk<EPI, bf16>(p, n, t0 + c, M, acc);
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (EPI == EPI_ARGMAX && ready) {
+    for (int j = threadIdx.x; j < ntile; j += blockDim.x) {
+      const int m = t0 + j;
+      if (m < M) {
+        float v = red_val[0][j];
+        int i = red_idx[0][j];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+          const float ov = red_val[w][j];
+          const int oi = red_idx[w][j];
+          if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+        }
+        p.part_val[(size_t)blockIdx.x * p.M_cap + m] = v;
+        p.part_idx[(size_t)blockIdx.x * p.M_cap + m] = i;
+      }
+    }
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+  }
+}
+
+}  // namespace tc
+}  // namespace ad

@@ -1,0 +1,426 @@
+// The small kernels around the GEMMs and attention: block planning (which tokens are fed at which
+// positions), embedding, LayerNorm, the arg-max reduction with the draft compare / first-mismatch decision,
+// the commit (cache-length advance / rollback), the input-guided draft policy of Algorithm 1, and the
+// planning of the drafter and encoder passes.
+#pragma once
+
+#include "ad_common.cuh"
+
+namespace ad {
+
+// Per-row decoding state and per-call block buffers, all resident in the workspace.
+struct DevState {
+  int* len;        // [B] accepted-prefix length = cached positions
+  int* last;       // [B] last accepted token ([BOS] at the start)
+  int* fin;        // [B] 1 once [EOS] was accepted or the row's cap was reached
+  int* maxlen;     // [B] per-row output cap
+  int* srclen;     // [B]
+  int* src;        // [B, max_src]
+  int* out_ids;    // [B, max_tgt]
+  int* drafts;     // [B, kmax]
+  int* pred;       // [B, kmax] greedy choices of the last verification
+  int* n_acc;      // [B] accepted count of the last verification (0 = nothing to commit)
+  int* stat_it;    // [B] iterations the row took part in
+  int* stat_acc;   // [B] tokens accepted
+  int* stat_off;   // [B] block sizes offered
+  int* loop_it;    // [1] iterations with at least one active row
+  int* status;     // [1] latched device error
+  int* all_fin;    // [1] 1 when every row is finished
+  int* cross_base; // [B] = b * max_src
+  int* gidx;       // [B * kmax] drafter: packed token holding mask position i of row b
+  int* enc_slot;   // [B * max_src] encoder: cross-K/V slot of packed source token m
+  int* user_k;     // [B] staging of caller-provided k / n
+  int* user_n;     // [B]
+  int* user_drafts;// [B, kmax]
+};
+
+enum DraftSource : int {
+  SRC_USER = 0,      // drafts and k come from the caller (ad_verify_block)
+  SRC_OVERRIDE = 1,  // k = min(cap, remaining); drafts = position-aligned stream
+  SRC_POLICY = 2,    // Algorithm 1: suffix match on the source
+  SRC_SIZES = 3,     // k = min(cap, remaining); drafts left untouched (the drafter fills them)
+  SRC_KEEP = 4       // k and drafts as they are (after the drafter); optional override on top
+};
+
+struct Dims {
+  int B, max_src, max_tgt, kmax;
+  int bos, pad, eos, mask;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Suffix match of Algorithm 1, line 3, for one row, executed by one warp.
+// o_0 = [BOS], o_t = out[t-1]; x_0 = [BOS], x_t = src[t-1], t <= n.  For q = 0, 1, ... counts the end
+// positions i with o[j-q..j] == x[i-q..i]; a unique one is the match, none means no match, several means
+// a longer suffix is tried.  Returns i or -1 (same value in every lane).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int tok_o(const int* out, int t, int bos) { return t == 0 ? bos : out[t - 1]; }
+
+__device__ int warp_suffix_match(const int* out, int j, const int* src, int n, int bos, int lane) {
+  for (int q = 0; q <= j; ++q) {
+    int count = 0, where = -1;
+    for (int i0 = q; i0 <= n; i0 += 32) {
+      const int i = i0 + lane;
+      bool ok = i <= n;
+      for (int t = 0; ok && t <= q; ++t) ok = tok_o(out, j - t, bos) == tok_o(src, i - t, bos);
+      const unsigned bal = __ballot_sync(0xffffffffu, ok);
+      if (bal) { count += __popc(bal); where = i0 + 31 - __clz(bal); }
+    }
+    if (count == 1) return where;
+    if (count == 0) return -1;
+  }
+  return -1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Chooses every row's block (size and drafted tokens) and lays the block tokens out as packed rows.
+// Decoder inputs of row b are (last accepted token, drafts[0..k-2]) at positions len .. len+k-1
+// (Eq. 6 / Eq. 7); a negative draft that would be fed is replaced by [PAD].
+// grid = 1, block = 256.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap, const int* override_stream,
+                      int override_stride, int override_len) {
+  __shared__ int s_k[256];
+  __shared__ int s_off[257];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int B = dm.B;
+
+  if (source == SRC_POLICY) {
+    for (int b = warp; b < B; b += 8) {
+      int k = 0;
+      const int len = st.len[b];
+      if (!st.fin[b] && len < st.maxlen[b]) {
+        const int n = st.srclen[b];
+        const int* src = st.src + (size_t)b * dm.max_src;
+        const int i = warp_suffix_match(st.out_ids + (size_t)b * dm.max_tgt, len, src, n, dm.bos, lane);
+        int* dr = st.drafts + (size_t)b * dm.kmax;
+        if (i >= 0) {
+          // draft = x_{i+1..n} followed by the [PAD] slot that matches nothing
+          k = n - i + 1;
+          k = min(k, min(k_cap, st.maxlen[b] - len));
+          for (int t = lane; t < k; t += 32) dr[t] = (i + 1 + t <= n) ? src[i + t] : -1;
+        } else {
+          k = 1;
+          if (lane == 0) dr[0] = -1;
+        }
+      }
+      if (lane == 0) s_k[b] = k;
+    }
+  } else {
+    for (int b = tid; b < B; b += 256) {
+      int k;
+      const int len = st.len[b];
+      if (source == SRC_USER) {
+        k = st.user_k[b];
+        if (k < 0 || k > dm.kmax || len + k > dm.max_tgt) { latch_error(st.status, AD_ERR_ARG); k = 0; }
+      } else if (source == SRC_KEEP) {
+        k = plan.seg_len[b];
+      } else {
+        k = (st.fin[b] || len >= st.maxlen[b]) ? 0 : min(k_cap, st.maxlen[b] - len);
+      }
+      s_k[b] = k;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < B; ++b) { s_off[b] = acc; acc += s_k[b]; }
+    s_off[B] = acc;
+    *plan.M = acc;
+  }
+  __syncthreads();
+  for (int b = warp; b < B; b += 8) {
+    const int k = s_k[b], off = s_off[b], len = st.len[b];
+    int* dr = st.drafts + (size_t)b * dm.kmax;
+    if (lane == 0) {
+      plan.seg_off[b] = off;
+      plan.seg_len[b] = k;
+      plan.key_base[b] = b * dm.max_tgt;
+    }
+    for (int i = lane; i < k; i += 32) {
+      if (source == SRC_USER) dr[i] = st.user_drafts[(size_t)b * dm.kmax + i];
+      if (override_stream && (source == SRC_OVERRIDE || source == SRC_KEEP))
+        dr[i] = (len + i < override_len) ? override_stream[(size_t)b * override_stride + len + i] : -1;
+    }
+    __syncwarp();
+    for (int i = lane; i < k; i += 32) {
+      const int m = off + i;
+      int tok = (i == 0) ? st.last[b] : dr[i - 1];
+      if (tok < 0) tok = dm.pad;
+      plan.tok_row[m] = b;
+      plan.tok_pos[m] = len + i;
+      plan.tok_id[m] = tok;
+      plan.kv_slot[m] = b * dm.max_tgt + len + i;
+      plan.att_n[m] = len + i + 1;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Drafter pass (Section 3.2.1): row b feeds ([BOS], accepted tokens, k x [MASK]) at positions 0 .. len+k
+// with no cache and unmasked attention.  blk is the verification plan holding k per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+plan_draft_kernel(DevState st, PassPlan blk, PassPlan plan, Dims dm) {
+  __shared__ int s_off[257];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int B = dm.B;
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < B; ++b) {
+      s_off[b] = acc;
+      const int k = blk.seg_len[b];
+      acc += k > 0 ? st.len[b] + 1 + k : 0;
+    }
+    s_off[B] = acc;
+    *plan.M = acc;
+  }
+  __syncthreads();
+  for (int b = warp; b < B; b += 8) {
+    const int k = blk.seg_len[b], len = st.len[b], off = s_off[b];
+    const int n = k > 0 ? len + 1 + k : 0;
+    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; }
+    for (int i = lane; i < n; i += 32) {
+      const int m = off + i;
+      plan.tok_row[m] = b;
+      plan.tok_pos[m] = i;
+      plan.tok_id[m] = (i == 0) ? dm.bos : (i <= len ? st.out_ids[(size_t)b * dm.max_tgt + i - 1] : dm.mask);
+      plan.kv_slot[m] = m;
+      plan.att_n[m] = n;
+    }
+    for (int i = lane; i < k; i += 32) st.gidx[blk.seg_off[b] + i] = off + len + 1 + i;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Encoder pass: row b feeds its src_len[b] source tokens (padding is simply not packed, and the per-row
+// key counts keep it out of every attention).  Also resets the decoding state of every row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
+  __shared__ int s_off[257];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int B = dm.B;
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < B; ++b) { s_off[b] = acc; acc += st.srclen[b]; }
+    *plan.M = acc;
+    *st.loop_it = 0;
+    *st.all_fin = 0;
+  }
+  for (int b = tid; b < B; b += 256) {
+    st.len[b] = 0; st.last[b] = dm.bos; st.fin[b] = 0; st.n_acc[b] = 0; st.maxlen[b] = dm.max_tgt;
+    st.stat_it[b] = 0; st.stat_acc[b] = 0; st.stat_off[b] = 0;
+    st.cross_base[b] = b * dm.max_src;
+  }
+  __syncthreads();
+  for (int b = warp; b < B; b += 8) {
+    const int n = st.srclen[b], off = s_off[b];
+    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; }
+    for (int i = lane; i < n; i += 32) {
+      const int m = off + i;
+      plan.tok_row[m] = b;
+      plan.tok_pos[m] = i;
+      plan.tok_id[m] = st.src[(size_t)b * dm.max_src + i];
+      plan.kv_slot[m] = m;
+      plan.att_n[m] = n;
+      st.enc_slot[m] = b * dm.max_src + i;
+    }
+  }
+}
+
+__global__ void set_maxlen_kernel(DevState st, Dims dm, const int* maxlen) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < dm.B) {
+    int v = maxlen[b];
+    if (v < 1 || v > dm.max_tgt) { latch_error(st.status, AD_ERR_ARG); v = max(1, min(v, dm.max_tgt)); }
+    st.maxlen[b] = v;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// y = emb[token] * sqrt(d) + PE[pos]  ->  FP32 residual stream and the GEMM-operand copy.
+// grid = M_cap, block = 128.
+// ---------------------------------------------------------------------------------------------
+template <typename WT, typename ActT>
+__global__ void __launch_bounds__(128)
+embed_kernel(PassPlan plan, const WT* __restrict__ emb, const float* __restrict__ pe, int d, float scale,
+             float* __restrict__ y, ActT* __restrict__ yb) {
+  const int m = blockIdx.x;
+  if (m >= *plan.M) return;
+  const int id = plan.tok_id[m], pos = plan.tok_pos[m];
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = to_f32(emb[(size_t)id * d + i]) * scale + pe[(size_t)pos * d + i];
+    y[(size_t)m * d + i] = v;
+    yb[(size_t)m * d + i] = from_f32<ActT>(v);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm (biased variance) of pre[m, :]; one warp per packed token.  grid = ceil(M_cap / 4), block = 128.
+// ---------------------------------------------------------------------------------------------
+template <typename ActT>
+__global__ void __launch_bounds__(128)
+layernorm_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, const float* __restrict__ g,
+                 const float* __restrict__ bta, int d, float eps, float* __restrict__ y, ActT* __restrict__ yb) {
+  const int m = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (m >= *M_ptr) return;
+  const float* x = pre + (size_t)m * d;
+  float s = 0.f;
+  for (int i = lane; i < d; i += 32) s += x[i];
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+  const float mean = s / (float)d;
+  float v = 0.f;
+  for (int i = lane; i < d; i += 32) { const float t = x[i] - mean; v = fmaf(t, t, v); }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  const float inv = rsqrtf(v / (float)d + eps);
+  for (int i = lane; i < d; i += 32) {
+    const float o = g[i] * ((x[i] - mean) * inv) + bta[i];
+    y[(size_t)m * d + i] = o;
+    yb[(size_t)m * d + i] = from_f32<ActT>(o);
+  }
+}
+
+// dst[j, :] = src[gidx[j], :] for j < *M_ptr.  grid = M_cap, block = 128.
+template <typename ActT>
+__global__ void __launch_bounds__(128)
+gather_rows_kernel(const int* __restrict__ M_ptr, const int* __restrict__ gidx, const ActT* __restrict__ src,
+                   ActT* __restrict__ dst, int d) {
+  const int j = blockIdx.x;
+  if (j >= *M_ptr) return;
+  const int s = gidx[j];
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(size_t)j * d + i] = src[(size_t)s * d + i];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Final arg-max over the per-tile partials of the fused projection, then the draft compare:
+//   c = first block position whose greedy choice differs from the draft (Section 3.1.1; definition of c
+//   in Section 3.2), n = c + 1 (the bifurcation token is kept), n = k when nothing differs, cut at the
+//   first accepted [EOS].  One CTA per row; warp 0 takes the decision with ballots.
+// to_drafts != 0: drafter mode, the choices are written as the row's drafts and nothing is compared.
+// grid = B, block = 128.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
+                     const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts) {
+  const int b = blockIdx.x;
+  const int k = blk.seg_len[b];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int* pred = (to_drafts ? st.drafts : st.pred) + (size_t)b * dm.kmax;
+  if (k == 0) {
+    if (tid == 0 && !to_drafts) st.n_acc[b] = 0;
+    return;
+  }
+  const int off = blk.seg_off[b];
+  for (int i = warp; i < k; i += 4) {
+    const int m = off + i;
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int t = lane; t < n_tiles; t += 32) {
+      const float ov = part_val[(size_t)t * M_cap + m];
+      const int oi = part_idx[(size_t)t * M_cap + m];
+      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+    }
+    if (lane == 0) pred[i] = idx;
+  }
+  if (to_drafts) return;
+  __syncthreads();
+  if (warp == 0) {
+    const int* dr = st.drafts + (size_t)b * dm.kmax;
+    int n = k;
+    bool found = false;
+    for (int i0 = 0; i0 < k && !found; i0 += 32) {
+      const int i = i0 + lane;
+      const bool mism = (i < k) && (dr[i] < 0 || pred[i] != dr[i]);
+      const unsigned bal = __ballot_sync(0xffffffffu, mism);
+      if (bal) { n = i0 + __ffs(bal); found = true; }
+    }
+    found = false;
+    for (int i0 = 0; i0 < n && !found; i0 += 32) {
+      const int i = i0 + lane;
+      const bool is_eos = (i < n) && (pred[i] == dm.eos);
+      const unsigned bal = __ballot_sync(0xffffffffu, is_eos);
+      if (bal) { n = i0 + __ffs(bal); found = true; }
+    }
+    if (lane == 0) st.n_acc[b] = n;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Commit: cache-length advance or rollback (Algorithm 1 lines 6-7).  n_in == null commits n_acc.
+// grid = 1, block = 256.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
+  __shared__ int s_active, s_allfin;
+  if (threadIdx.x == 0) { s_active = 0; s_allfin = 1; }
+  __syncthreads();
+  for (int b = threadIdx.x; b < dm.B; b += 256) {
+    const int nacc = st.n_acc[b];
+    int n = n_in ? n_in[b] : nacc;
+    int len = st.len[b];
+    if (n > nacc || (n < 0 && -n > len)) {
+      latch_error(st.status, AD_ERR_ARG);
+      n = 0;
+    }
+    if (n > 0) {
+      const int* pred = st.pred + (size_t)b * dm.kmax;
+      int* out = st.out_ids + (size_t)b * dm.max_tgt;
+      for (int i = 0; i < n; ++i) out[len + i] = pred[i];
+      len += n;
+      st.len[b] = len;
+      st.last[b] = pred[n - 1];
+      if (pred[n - 1] == dm.eos || len >= st.maxlen[b]) st.fin[b] = 1;
+      st.stat_acc[b] += n;
+    } else if (n < 0) {
+      len += n;
+      st.len[b] = len;
+      st.last[b] = len > 0 ? st.out_ids[(size_t)b * dm.max_tgt + len - 1] : dm.bos;
+      st.fin[b] = 0;
+    }
+    if (nacc > 0) {
+      st.stat_it[b] += 1;
+      st.stat_off[b] += blk.seg_len[b];
+      atomicOr(&s_active, 1);
+    }
+    st.n_acc[b] = 0;
+    if (!st.fin[b]) atomicAnd(&s_allfin, 0);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (s_active) *st.loop_it += 1;
+    *st.all_fin = s_allfin;
+  }
+}
+
+// Copies the block results to caller-visible arrays (device pointers).  grid = B, block = 64.
+__global__ void export_block_kernel(DevState st, Dims dm, int* argmax_out, int* n_out, int* drafts_out, int* k_out,
+                                    PassPlan blk) {
+  const int b = blockIdx.x;
+  if (argmax_out)
+    for (int i = threadIdx.x; i < dm.kmax; i += blockDim.x) argmax_out[(size_t)b * dm.kmax + i] = st.pred[(size_t)b * dm.kmax + i];
+  if (drafts_out)
+    for (int i = threadIdx.x; i < dm.kmax; i += blockDim.x) drafts_out[(size_t)b * dm.kmax + i] = st.drafts[(size_t)b * dm.kmax + i];
+  if (threadIdx.x == 0) {
+    if (n_out) n_out[b] = st.n_acc[b];
+    if (k_out) k_out[b] = blk.seg_len[b];
+  }
+}
+
+// FP32 copy of an activation buffer (debug).  grid-stride.
+template <typename ActT>
+__global__ void to_f32_kernel(const ActT* __restrict__ src, float* __restrict__ dst, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = to_f32(src[i]);
+}
+
+}  // namespace ad
