@@ -164,6 +164,14 @@ int ad_verify_block(ad_handle* h, const int32_t* drafts, const int32_t* k, int32
  * No data moves on rollback: stale cache slots are overwritten by later blocks. */
 int ad_commit(ad_handle* h, const int32_t* n, int32_t on_host);
 
+/* Teacher forcing (Eq. 1: scoring with a known prefix): declares tokens[b][0 .. n_b) to be the next n_b output
+ * tokens of row b after an ad_verify_block, whatever the verifier predicted.  tokens [B, kmax], n [B] with
+ * 0 <= n_b <= k_b of that block.  The cache stays consistent only if the block fed exactly these tokens, so the
+ * call requires tokens[b][i] == drafts[b][i] for i < n_b - 1 (else AD_ERR_ARG, row unchanged).  Sets
+ * len_b += n_b and the last token to tokens[b][n_b-1]; the row finishes on [EOS] or at its cap.  Used to walk
+ * the library along a reference trajectory position by position. */
+int ad_force_commit(ad_handle* h, const int32_t* tokens, const int32_t* n, int32_t on_host);
+
 /* Whole decoding loop (Algorithm 1; Section 3.2 loop "until [EOS] or the maximal length").  Encodes src,
  * then iterates draft -> verify -> commit on the device until every row has finished.  out [B, out_stride]
  * receives the tokens (an [EOS] included when produced), out_len [B] their count.  stats may be NULL.

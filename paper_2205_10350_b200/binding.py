@@ -20,7 +20,7 @@ AD_MODE_IAD, AD_MODE_GAD = 0, 1
 
 EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
-    "ad_verify_block", "ad_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync",
+    "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync",
     "ad_debug_logits", "ad_debug_encoder_memory", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
     "ad_linear",
 ]
@@ -79,6 +79,7 @@ def load():
         "ad_encode": (C.c_int, [vp, vp, i32, vp, i32, i32]),
         "ad_verify_block": (C.c_int, [vp, vp, vp, vp, vp, i32]),
         "ad_commit": (C.c_int, [vp, vp, i32]),
+        "ad_force_commit": (C.c_int, [vp, vp, vp, i32]),
         "ad_generate": (C.c_int, [vp, vp, i32, vp, i32, C.POINTER(GenOpts), vp, i32, vp, C.POINTER(Stats), i32]),
         "ad_draft_block": (C.c_int, [vp, i32, vp, vp, i32]),
         "ad_get_state": (C.c_int, [vp, vp, vp, vp]),
@@ -210,6 +211,13 @@ class AggressiveDecoder:
         else:
             n = _i32(n)
             self._check(self.lib.ad_commit(self.h, n.ctypes.data, 1), self.h)
+
+    def force_commit(self, tokens, n):
+        t = np.full((self.B, self.kmax), -1, np.int32)
+        tokens = np.asarray(tokens, np.int32)
+        t[:, : tokens.shape[1]] = tokens
+        n = _i32(n)
+        self._check(self.lib.ad_force_commit(self.h, t.ctypes.data, n.ctypes.data, 1), self.h)
 
     def draft_block(self, k_cap):
         d = np.zeros((self.B, self.kmax), np.int32)

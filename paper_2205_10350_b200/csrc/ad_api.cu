@@ -721,6 +721,19 @@ extern "C" int ad_commit(ad_handle* h, const int32_t* n, int32_t on_host) {
   return AD_OK;
 }
 
+extern "C" int ad_force_commit(ad_handle* h, const int32_t* tokens, const int32_t* n, int32_t on_host) {
+  if (!h) return AD_ERR_ARG;
+  if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_force_commit before ad_encode");
+  if (!tokens || !n) return fail(h, AD_ERR_ARG, "tokens or n is null");
+  AD_CUDA(h, cudaMemcpyAsync(h->st.user_drafts, tokens, sizeof(int) * (size_t)h->B * h->cfg.kmax, to_dev(on_host), h->stream));
+  AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, n, sizeof(int) * h->B, to_dev(on_host), h->stream));
+  h->launches++;
+  force_commit_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, h->st.user_drafts, h->st.user_n);
+  AD_CUDA(h, cudaGetLastError());
+  if (on_host) return read_status(h);
+  return AD_OK;
+}
+
 extern "C" int ad_draft_block(ad_handle* h, int32_t k_cap, int32_t* drafts, int32_t* k, int32_t on_host) {
   if (!h) return AD_ERR_ARG;
   if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_draft_block before ad_encode");

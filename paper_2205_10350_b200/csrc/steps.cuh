@@ -402,6 +402,29 @@ commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
   }
 }
 
+// Teacher-forced commit: the caller supplies the accepted tokens.  grid = 1, block = 256.
+__global__ void __launch_bounds__(256)
+force_commit_kernel(DevState st, PassPlan blk, Dims dm, const int* tokens, const int* n_in) {
+  for (int b = threadIdx.x; b < dm.B; b += 256) {
+    const int n = n_in[b], k = blk.seg_len[b];
+    const int* tk = tokens + (size_t)b * dm.kmax;
+    const int* dr = st.drafts + (size_t)b * dm.kmax;
+    bool ok = n >= 0 && n <= k;
+    for (int i = 0; ok && i + 1 < n; ++i) ok = tk[i] == dr[i];
+    if (!ok) { latch_error(st.status, AD_ERR_ARG); continue; }
+    if (n > 0) {
+      int len = st.len[b];
+      int* out = st.out_ids + (size_t)b * dm.max_tgt;
+      for (int i = 0; i < n; ++i) out[len + i] = tk[i];
+      len += n;
+      st.len[b] = len;
+      st.last[b] = tk[n - 1];
+      if (tk[n - 1] == dm.eos || len >= st.maxlen[b]) st.fin[b] = 1;
+    }
+    st.n_acc[b] = 0;
+  }
+}
+
 // Copies the block results to caller-visible arrays (device pointers).  grid = B, block = 64.
 __global__ void export_block_kernel(DevState st, Dims dm, int* argmax_out, int* n_out, int* drafts_out, int* k_out,
                                     PassPlan blk) {

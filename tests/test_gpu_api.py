@@ -1,0 +1,111 @@
+"""Edge cases and error behaviour of the C ABI on the device (no faults: every bad input is turned into an
+error code by the host or by the kernels' own checks)."""
+import numpy as np
+import pytest
+
+from oracle import ad_oracle as O
+from paper_2205_10350_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def setup():
+    shape = synth.ModelShape("edge", 64, 2, 128, 50, 1, 1, "fp32")
+    w = synth.make_weights(shape, 0, std=0.1)
+    dec = binding.AggressiveDecoder(shape, w, max_batch=4, max_src=10, max_tgt=12, kmax=6)
+    om = O.Model(shape, w, max_pos=16)
+    return dec, om
+
+
+def test_call_order_and_capacity_errors(setup):
+    dec, om = setup
+    fresh = binding.AggressiveDecoder(dec.shape, synth.make_weights(dec.shape, 0, std=0.1), max_batch=2, max_src=10,
+                                      max_tgt=12, kmax=6)
+    fresh.B = 1
+    with pytest.raises(binding.AdError) as e:
+        fresh.verify_block(np.zeros((1, 6), np.int32), [1])
+    assert e.value.code == binding.AD_ERR_STATE
+    with pytest.raises(binding.AdError) as e:
+        fresh.encode(np.full((3, 10), 5, np.int32), [3, 3, 3])
+    assert e.value.code == binding.AD_ERR_CAPACITY
+    with pytest.raises(binding.AdError) as e:
+        fresh.encode(np.full((1, 10), 5, np.int32), [11])
+    assert e.value.code == binding.AD_ERR_CAPACITY
+    with pytest.raises(binding.AdError) as e:
+        fresh.encode(np.full((1, 10), 5, np.int32), [0])
+    assert e.value.code == binding.AD_ERR_ARG
+    with pytest.raises(binding.AdError) as e:
+        fresh.generate(np.full((1, 10), 5, np.int32), [4], mode="GAD", k=2, run_drafter=True)
+    assert e.value.code == binding.AD_ERR_STATE
+    with pytest.raises(binding.AdError) as e:
+        fresh.generate(np.full((1, 10), 5, np.int32), [4], mode="IAD", k=7)
+    assert e.value.code == binding.AD_ERR_ARG
+
+
+def test_idle_rows_ragged_blocks_commit_and_rollback(setup):
+    dec, om = setup
+    src = np.array([[5, 6, 7, 8, 9, 10, 11, 12, 13, 14]] * 3, np.int32)
+    lens = np.array([10, 4, 7], np.int32)
+    dec.encode(src, lens)
+    states = [om.state(src[b, : lens[b]], cap=12) for b in range(3)]
+    drafts = np.array([[20, 21, 22, 23, 24, 25], [30, -1, -1, -1, -1, -1], [0] * 6], np.int32)
+    ks = np.array([6, 1, 0], np.int32)                      # full block, single step, idle row
+    am, n = dec.verify_block(drafts, ks)
+    assert n[2] == 0
+    for b in (0, 1):
+        res = states[b].verify_block(0, drafts[b, : ks[b]])
+        assert np.array_equal(am[b, : ks[b]], res["pred"]) and n[b] == res["n"]
+    # committing more than was accepted is refused and leaves the row alone
+    with pytest.raises(binding.AdError) as e:
+        dec.commit([int(n[0]) + 1, 0, 0])
+    assert e.value.code == binding.AD_ERR_ARG
+    ln, last, fin = dec.state()
+    assert (ln == 0).all()
+    am, n = dec.verify_block(drafts, ks)
+    dec.commit()                                             # NULL = commit what was accepted
+    ln, last, fin = dec.state()
+    assert ln[0] == n[0] and ln[1] == n[1] and ln[2] == 0
+    assert last[0] == am[0, n[0] - 1]
+    # commit without a fresh verification is a no-op
+    dec.commit()
+    ln2, _, _ = dec.state()
+    assert np.array_equal(ln, ln2)
+    # rollback by one and re-verify: same prediction as before at that position
+    if ln[0] >= 1:
+        dec.commit([-1, 0, 0])
+        ln3, last3, _ = dec.state()
+        assert ln3[0] == ln[0] - 1
+    with pytest.raises(binding.AdError):
+        dec.commit([-50, 0, 0])                              # cannot roll back more than was committed
+    # k beyond the cache capacity is refused by the device-side check
+    with pytest.raises(binding.AdError) as e:
+        dec.verify_block(drafts, [7, 0, 0])
+    assert e.value.code == binding.AD_ERR_ARG
+
+
+def test_maximum_sizes_and_cap_reached(setup):
+    dec, om = setup
+    src = np.full((4, 10), 6, np.int32)
+    src[:, ::2] = 9
+    lens = np.array([10, 10, 1, 10], np.int32)
+    outs, stats = dec.generate(src, lens, mode="IAD", k=6, max_len=[12, 1, 12, 5])
+    for b, cap in enumerate([12, 1, 12, 5]):
+        g, _ = om.state(src[b, : lens[b]], cap=12).greedy(cap)
+        assert np.array_equal(outs[b], g)
+    ln, _, fin = dec.state()
+    assert (fin == 1).all()
+
+
+def test_teacher_forcing_rejects_inconsistent_tokens(setup):
+    dec, om = setup
+    src = np.full((1, 10), 6, np.int32)
+    dec.encode(src, [5])
+    dec.verify_block(np.array([[20, 21, 22, -1, -1, -1]], np.int32), [3])
+    with pytest.raises(binding.AdError) as e:
+        dec.force_commit(np.array([[20, 33, 40]], np.int32), [3])     # second token was not what the block fed
+    assert e.value.code == binding.AD_ERR_ARG
+    dec.verify_block(np.array([[20, 21, 22, -1, -1, -1]], np.int32), [3])
+    dec.force_commit(np.array([[20, 21, 40]], np.int32), [3])
+    ln, last, _ = dec.state()
+    assert ln[0] == 3 and last[0] == 40

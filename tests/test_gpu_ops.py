@@ -1,0 +1,79 @@
+"""Operator-level parity through the C ABI: the two GEMM kernels and the fused projection + arg-max against
+the CPU checker's linear map, at sizes that span several tiles and a ragged tail."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ad_oracle as O
+from paper_2205_10350_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+OPS = O.Ops("f32")
+
+
+def _data(M, K, N, bf16, seed=0):
+    r = np.random.default_rng(seed)
+    x = r.standard_normal((M, K)).astype(np.float32)
+    W = (r.standard_normal((N, K)) * 0.1).astype(np.float32)
+    b = r.standard_normal(N).astype(np.float32)
+    if bf16:
+        x, W = synth.round_to_bf16(x), synth.round_to_bf16(W)
+    return x, W, b
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 128, 128), (5, 128, 130), (33, 96, 1000), (17, 512, 257)])
+def test_fp32_linear(M, K, N):
+    x, W, b = _data(M, K, N, False)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    y = binding.linear(torch.tensor(x, device=DEV), torch.tensor(W, device=DEV), torch.tensor(b, device=DEV), st)
+    ref = OPS.linear(x, W.T.copy(), b)
+    assert np.abs(y.cpu().numpy() - ref).max() < 1e-4
+    assert int(st.item()) == 0
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 64, 128), (16, 64, 128), (64, 512, 1536), (25, 1024, 300), (200, 512, 512),
+                                   (256, 2048, 640), (7, 4096, 128)])
+def test_bf16_tensor_core_linear(M, K, N):
+    """Inputs are BF16-exact, the accumulator is FP32: only the summation order differs from the checker."""
+    x, W, b = _data(M, K, N, True)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    y = binding.linear(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(W, device=DEV).bfloat16(),
+                       torch.tensor(b, device=DEV), st)
+    ref = OPS.linear(x, W.T.copy(), b)
+    assert np.abs(y.cpu().numpy() - ref).max() < 2e-4 * max(1.0, np.abs(ref).max())
+    assert int(st.item()) == 0
+
+
+@pytest.mark.parametrize("bf16,M,d,V", [(False, 9, 128, 1000), (True, 40, 512, 32000), (True, 64, 1024, 4100),
+                                        (True, 1, 512, 32000), (True, 130, 256, 2048)])
+def test_projection_with_fused_argmax(bf16, M, d, V):
+    r = np.random.default_rng(4)
+    x = r.standard_normal((M, d)).astype(np.float32)
+    E = (r.standard_normal((V, d)) * 0.02).astype(np.float32)
+    if bf16:
+        x, E = synth.round_to_bf16(x), synth.round_to_bf16(E)
+    tx, tE = torch.tensor(x, device=DEV), torch.tensor(E, device=DEV)
+    if bf16:
+        tx, tE = tx.bfloat16(), tE.bfloat16()
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    got = binding.vocab_argmax(tx, tE, st).cpu().numpy()
+    lg = OPS.linear(x, E.T.copy(), None)
+    for m in range(M):
+        i1, v1, i2, v2 = OPS.top2(lg[m])
+        if v1 - v2 > 1e-4:
+            assert got[m] == i1
+        else:
+            assert got[m] in (i1, i2)
+    assert int(st.item()) == 0
+
+
+def test_argmax_ties_go_to_the_lowest_id():
+    d, V, M = 128, 700, 3
+    x = np.ones((M, d), np.float32)
+    E = np.zeros((V, d), np.float32)
+    E[[650, 131, 400]] = 0.5           # three identical best rows in different 128-row tiles
+    got = binding.vocab_argmax(torch.tensor(x, device=DEV), torch.tensor(E, device=DEV)).cpu().numpy()
+    assert (got == 131).all()
+    got = binding.vocab_argmax(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(E, device=DEV).bfloat16()).cpu().numpy()
+    assert (got == 131).all()

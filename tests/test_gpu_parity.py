@@ -1,0 +1,238 @@
+"""Parity of the CUDA path with the CPU checker on the five workload recipes, through the C ABI.
+
+Bars: token ids, accepted lengths and cache lengths exact wherever the checker's top-1/top-2 score gap
+exceeds 0.1; scores within 1e-3 (FP32 model) / 5e-2 (BF16 models) max-abs.
+"""
+import numpy as np
+import pytest
+
+from oracle import ad_oracle as O
+from paper_2205_10350_b200 import binding, synth
+from tests import parity_util as P
+
+pytestmark = pytest.mark.gpu
+TOL_FP32, TOL_BF16 = 1e-3, 5e-2
+
+
+def make(shape, wl_batch, max_src, max_tgt, kmax, drafter=False, std=0.02):
+    w = synth.make_weights(shape, 0, std=std)
+    wn = synth.make_weights(shape, 1, std=std) if drafter else None
+    dec = binding.AggressiveDecoder(shape, w, wn, max_batch=wl_batch, max_src=max_src, max_tgt=max_tgt, kmax=kmax)
+    om = O.Model(shape, w, max_pos=max(max_src, max_tgt + 1))
+    on = O.Model(shape, wn, max_pos=max(max_src, max_tgt + 1)) if drafter else None
+    return dec, om, on
+
+
+# ------------------------------------------------------------------------------------------ workload 1
+@pytest.fixture(scope="module")
+def tiny():
+    return make(synth.TINY, 1, 16, 24, 17, drafter=True)
+
+
+def test_tiny_encoder_memory(tiny):
+    dec, om, _ = tiny
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    dec.encode(src, lens)
+    mem = dec.debug_encoder_memory(0, int(lens[0]))
+    assert np.abs(mem - om.state(src[0, :lens[0]]).memory()).max() < 1e-4
+
+
+def test_tiny_lockstep_source_copy_drafts(tiny):
+    dec, om, _ = tiny
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    stream = np.concatenate([src[0, :16], np.full(16, -1, np.int32)])
+    tot = P.lockstep(dec, om, src, lens, [stream], 17, [24], TOL_FP32)
+    assert tot["tokens"] == 24 and tot["worst_logit_err"] < TOL_FP32
+
+
+def test_tiny_input_guided_generate_is_identical_to_greedy(tiny):
+    dec, om, _ = tiny
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    st = om.state(src[0, :lens[0]])
+    g, margin = st.greedy(24)
+    ref_out, ref_tr = st.iad(17, 24)
+    for graph in (False, True):
+        outs, stats = dec.generate(src, lens, mode="IAD", k=17, max_len=[24], use_graph=graph)
+        assert np.array_equal(outs[0], g)
+        assert stats["iterations"] == ref_tr["iterations"] and stats["offered"] == ref_tr["offered"]
+        assert stats["accepted"] == len(g)
+    outs, stats = dec.generate(src, lens, mode="IAD", k=1, max_len=[24])      # k = 1 is greedy decoding
+    assert np.array_equal(outs[0], g) and stats["iterations"] == len(g)
+
+
+def test_tiny_generalized_mode_with_real_drafter(tiny):
+    dec, om, on = tiny
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    st = om.state(src[0, :lens[0]])
+    g, _ = st.greedy(24)
+    ref_out, ref_tr = st.gad(on, 5, 24)
+    outs, stats = dec.generate(src, lens, mode="GAD", k=5, max_len=[24], run_drafter=True)
+    assert np.array_equal(outs[0], g)
+    assert stats["iterations"] == ref_tr["iterations"]
+    # drafter block alone, at the start of decoding
+    dec.encode(src, lens)
+    d, k = dec.draft_block(5)
+    ref_d, ref_m = on.nar_draft(on.encode_memory(src[0, :lens[0]]), [0], 5)
+    assert k[0] == 5
+    for i in range(5):
+        assert d[0, i] == ref_d[i] or ref_m[i] <= P.MARGIN
+
+
+# A model with larger weights decodes to varied text, which exercises suffix matching, rollback and EOS.
+@pytest.mark.parametrize("seed_std", [0.08, 0.15])
+def test_varied_fp32_model_all_modes(seed_std):
+    shape = synth.ModelShape("vary", 64, 2, 128, 40, 1, 2, "fp32")
+    dec, om, on = make(shape, 3, 12, 30, 13, drafter=True, std=seed_std)
+    r = np.random.default_rng(5)
+    lens = np.array([12, 7, 9], np.int32)
+    src = np.full((3, 12), synth.PAD, np.int32)
+    for b in range(3):
+        src[b, : lens[b]] = r.integers(4, 40, size=lens[b])
+    max_len = np.array([30, 18, 25], np.int32)
+    greedy = [om.state(src[b, : lens[b]]).greedy(int(max_len[b])) for b in range(3)]
+    outs, stats = dec.generate(src, lens, mode="IAD", k=13, max_len=max_len)
+    iters = 0
+    for b in range(3):
+        assert P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"IAD row {b}") is None
+        iters += om.state(src[b, : lens[b]]).iad(13, int(max_len[b]))[1]["iterations"]
+    assert stats["row_iterations"] == iters
+    outs, _ = dec.generate(src, lens, mode="GAD", k=4, max_len=max_len, run_drafter=True)
+    for b in range(3):
+        assert P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"GAD row {b}") is None
+    streams = np.full((3, 30), 5, np.int32)
+    for b in range(3):
+        g = greedy[b][0]
+        streams[b, : len(g)] = np.where(r.random(len(g)) < 0.7, g, 6)
+    outs, stats = dec.generate(src, lens, mode="GAD", k=6, max_len=max_len, draft_override=streams)
+    for b in range(3):
+        assert P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"stream row {b}") is None
+    tot = P.lockstep(dec, om, src, lens, list(streams), 6, max_len, TOL_FP32)
+    assert tot["flipped"] == 0
+
+
+# ------------------------------------------------------------------------------------------ small BF16
+def test_mini_bf16_lockstep_and_generate():
+    shape = synth.MINI_BF16
+    dec, om, on = make(shape, 4, 20, 24, 16, drafter=True)
+    wl = synth.Workload(9, shape, "IAD", 4, 1, 9, 20, 0, 16, 0.8, True)
+    src, lens = synth.make_sources(wl)
+    max_len = np.minimum(lens, 24)
+    greedy = [om.state(src[b, : lens[b]]).greedy(int(max_len[b])) for b in range(4)]
+    g = np.full((4, 24), synth.PAD, np.int32)
+    for b in range(4):
+        g[b, : len(greedy[b][0])] = greedy[b][0]
+    streams = synth.corrupt_stream(g, max_len, 0.8, shape.vocab, 9)
+    tot = P.lockstep(dec, om, src, lens, list(streams), 16, max_len, TOL_BF16)
+    assert tot["tokens"] == int(sum(len(x[0]) for x in greedy))
+    outs, _ = dec.generate(src, lens, mode="IAD", k=16, max_len=max_len, draft_override=streams)
+    for b in range(4):
+        P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"row {b}")
+    outs, _ = dec.generate(src, lens, mode="GAD", k=8, max_len=max_len, run_drafter=True)
+    for b in range(4):
+        P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"GAD row {b}")
+
+
+# ------------------------------------------------------------------------------------------ workloads 2, 3
+@pytest.fixture(scope="module")
+def base_weights():
+    return synth.make_weights(synth.BASE, 0)
+
+
+def _greedy_streams(om, src, lens, max_len, agreement, wl_index, vocab):
+    B = len(lens)
+    greedy = [om.state(src[b, : lens[b]]).greedy(int(max_len[b])) for b in range(B)]
+    g = np.full((B, int(max(max_len))), synth.PAD, np.int32)
+    gl = np.zeros(B, np.int32)
+    for b in range(B):
+        g[b, : len(greedy[b][0])] = greedy[b][0]
+        gl[b] = len(greedy[b][0])
+    return greedy, synth.corrupt_stream(g, gl, agreement, vocab, wl_index)
+
+
+def test_workload2_base_batch1(base_weights):
+    wl = synth.WORKLOADS[2]
+    dec = binding.AggressiveDecoder(synth.BASE, base_weights, max_batch=1, max_src=40, max_tgt=40, kmax=40)
+    om = O.Model(synth.BASE, base_weights, max_pos=64)
+    for sent in range(3):
+        src, lens = synth.make_sources(wl, sent)
+        max_len = synth.max_out_lens(wl, lens)
+        greedy, streams = _greedy_streams(om, src, lens, max_len, wl.agreement, wl.index, wl.shape.vocab)
+        kcap = min(wl.k, dec.kmax)       # outputs are at most 40 tokens here, so the cap of 64 never binds
+        tot = P.lockstep(dec, om, src, lens, list(streams), kcap, max_len, TOL_BF16)
+        assert tot["tokens"] == len(greedy[0][0])
+        outs, stats = dec.generate(src, lens, mode="IAD", k=kcap, max_len=max_len, draft_override=streams)
+        P.check_free_run(outs[0], greedy[0][0], greedy[0][1], f"sentence {sent}")
+        assert 1 <= stats["iterations"] <= len(outs[0])
+
+
+def test_workload3_base_batch32(base_weights):
+    wl = synth.WORKLOADS[3]
+    dec = binding.AggressiveDecoder(synth.BASE, base_weights, max_batch=32, max_src=64, max_tgt=64, kmax=64)
+    om = O.Model(synth.BASE, base_weights, max_pos=80)
+    src, lens = synth.make_sources(wl)
+    max_len = synth.max_out_lens(wl, lens)
+    greedy, streams = _greedy_streams(om, src, lens, max_len, wl.agreement, wl.index, wl.shape.vocab)
+    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, max_steps=2)
+    assert tot["steps"] == 2
+    outs, stats = dec.generate(src, lens, mode="IAD", k=wl.k, max_len=max_len, draft_override=streams)
+    for b in range(wl.batch):
+        P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"row {b}")
+    ln, _, fin = dec.state()
+    assert (fin == 1).all() and all(ln[b] == len(outs[b]) for b in range(wl.batch))
+
+
+# ------------------------------------------------------------------------------------------ workloads 4, 5
+def _drafter_parity(dec, on, src, lens, k):
+    """Drafter block at the start of decoding against the checker's drafter forward."""
+    d, kk = dec.draft_block(k)
+    for b in range(len(lens)):
+        ref_d, ref_m = on.nar_draft(on.encode_memory(src[b, : lens[b]]), [0], k)
+        assert kk[b] == k
+        for i in range(k):
+            assert d[b, i] == ref_d[i] or ref_m[i] <= P.MARGIN, (b, i, d[b, i], ref_d[i], ref_m[i])
+
+
+def test_workload4_big_generalized():
+    wl = synth.WORKLOADS[4]
+    dec, om, on = make(synth.BIG, 1, 50, 50, 25, drafter=True)
+    src, lens = synth.make_sources(wl, 0)
+    max_len = synth.max_out_lens(wl, lens)
+    greedy, streams = _greedy_streams(om, src, lens, max_len, wl.agreement, wl.index, wl.shape.vocab)
+    dec.encode(src, lens)
+    _drafter_parity(dec, on, src, lens, wl.k)
+    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, max_steps=3)
+    assert tot["steps"] >= 1
+    outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=max_len, draft_override=streams, run_drafter=True)
+    P.check_free_run(outs[0], greedy[0][0], greedy[0][1], "big")
+
+
+def test_workload5_base_long_source_batch8(base_weights):
+    wl = synth.WORKLOADS[5]
+    wn = synth.make_weights(synth.BASE, 1)
+    dec = binding.AggressiveDecoder(synth.BASE, base_weights, wn, max_batch=8, max_src=400, max_tgt=80, kmax=25)
+    om = O.Model(synth.BASE, base_weights, max_pos=401)
+    on = O.Model(synth.BASE, wn, max_pos=401)
+    src, lens = synth.make_sources(wl)
+    max_len = synth.max_out_lens(wl, lens)
+    # a perfect stream is not needed for lock-step: take uniform random drafts mixed with the checker's own
+    # first greedy tokens so that several positions are accepted
+    states = [om.state(src[b, : lens[b]], cap=80) for b in range(2)]
+    dec.encode(src, lens)
+    mem = dec.debug_encoder_memory(1, int(lens[1]))
+    assert np.abs(mem - states[1].memory()).max() < TOL_BF16
+    _drafter_parity(dec, on, src[:1], lens[:1], 5)
+    g8 = [st.greedy(8) for st in states]
+    streams = np.full((8, 80), 7, np.int32)
+    for b in range(2):
+        streams[b, : len(g8[b][0])] = g8[b][0]
+        streams[b, 5] = 9
+    # only rows 0 and 1 are checked against the checker (the others run but would cost minutes on the CPU)
+    dec2_src, dec2_lens = src[:2], lens[:2]
+    tot = P.lockstep(dec, om, dec2_src, dec2_lens, list(streams[:2]), wl.k, [80, 80], TOL_BF16, max_steps=2)
+    assert tot["steps"] == 2
+    # full batch, free running, repeated rollbacks (agreement 0.6 on a random stream): the loop must terminate
+    outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=np.full(8, 12, np.int32), draft_override=streams,
+                               run_drafter=True)
+    assert all(1 <= len(o) <= 12 for o in outs)
+    for b in range(2):
+        P.check_free_run(outs[b][:8], g8[b][0][:len(outs[b][:8])], g8[b][1], f"row {b}")
