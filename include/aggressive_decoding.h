@@ -115,6 +115,7 @@ typedef struct ad_stats {
   int64_t offered;         /* sum of block sizes offered */
   float device_ms;         /* device time of the decode loop (CUDA events), encoders excluded */
   float encode_ms;         /* device time of the encoder pass(es) */
+  int64_t kernel_launches; /* kernels of this library launched by the call (a graph replay counts its kernel nodes) */
 } ad_stats;
 
 typedef struct ad_handle ad_handle;

@@ -48,7 +48,8 @@ class GenOpts(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("iterations", C.c_int64), ("row_iterations", C.c_int64), ("accepted", C.c_int64),
-                ("offered", C.c_int64), ("device_ms", C.c_float), ("encode_ms", C.c_float)]
+                ("offered", C.c_int64), ("device_ms", C.c_float), ("encode_ms", C.c_float),
+                ("kernel_launches", C.c_int64)]
 
 
 class AdError(RuntimeError):
@@ -246,7 +247,7 @@ class AggressiveDecoder:
         return t.cpu().numpy()
 
     def generate(self, src, src_len, mode="IAD", k=1, max_len=None, draft_override=None, run_drafter=False,
-                 sync_every=0, use_graph=True):
+                 sync_every=0, use_graph=True, out=None, out_len=None):
         """Host-array form of ad_generate.  Returns (list of per-row outputs, stats dict)."""
         src, src_len = _i32(src), _i32(src_len)
         B = src.shape[0]
@@ -265,8 +266,10 @@ class AggressiveDecoder:
         opts.run_drafter = int(run_drafter)
         opts.sync_every = sync_every
         opts.use_graph = int(use_graph)
-        out = np.zeros((B, self.max_tgt), np.int32)
-        out_len = np.zeros(B, np.int32)
+        if out is None:
+            out = np.zeros((B, self.max_tgt), np.int32)
+        if out_len is None:
+            out_len = np.zeros(B, np.int32)
         st = Stats()
         self._check(self.lib.ad_generate(self.h, src.ctypes.data, src.shape[1], src_len.ctypes.data, B,
                                          C.byref(opts), out.ctypes.data, out.shape[1], out_len.ctypes.data,

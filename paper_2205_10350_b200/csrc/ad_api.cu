@@ -865,6 +865,7 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
     stats->iterations = buf[3 * B];
     cudaEventElapsedTime(&stats->encode_ms, h->ev0, h->ev1);
     cudaEventElapsedTime(&stats->device_ms, h->ev1, h->ev2);
+    stats->kernel_launches = h->launches;
   }
   return read_status(h);
 }

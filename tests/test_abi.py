@@ -75,7 +75,7 @@ def test_workspace_query_and_config_checks(lib):
 def test_struct_layouts():
     assert C.sizeof(binding.ModelCfg) == 17 * 4
     assert C.sizeof(binding.GenOpts) == 40
-    assert C.sizeof(binding.Stats) == 40
+    assert C.sizeof(binding.Stats) == 48
 
 
 def test_null_handle_calls_are_rejected(lib):
