@@ -213,6 +213,31 @@ size_t ad_vocab_argmax_scratch_bytes(int32_t vocab, int32_t M);
 int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d, int32_t vocab,
                     int32_t* argmax, void* scratch, size_t scratch_bytes, int32_t* status, void* stream);
 
+/* (No counterpart in the paper: this entry point exists for the sake of callers, not of the method.)
+ * Same computation and arguments as ad_vocab_argmax, but the caller provides no scratch buffer: the per-tile
+ * partial maxima live in a fixed array that is part of the library image itself.
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the point of the call -- for example a
+ * plug-in running inside a host application that owns the whole memory pool, a real-time or signal-handler-
+ * like context where cudaMalloc's implicit synchronisation is unacceptable, or a process whose allocator has
+ * already handed every byte to someone else.  Such callers still pass their inputs (x, emb) and the output
+ * (argmax); the library neither calls cudaMalloc/cudaFree nor any routine that allocates on their behalf.
+ *
+ * Limits and rules
+ *   - The built-in array is AD_STATIC_SCRATCH_BYTES (1 MiB) per GPU; every GPU that loads the library carries
+ *     it until the process exits.  A problem needs ad_vocab_argmax_scratch_bytes(vocab, M) bytes; larger
+ *     problems are refused with AD_ERR_CAPACITY (ad_last_error(NULL) then says how much was needed).
+ *     1 MiB covers, e.g., vocab 32000 with M up to 256 rows, or vocab 65536 with M up to 256.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current) and remembers it.  Make that first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left there.  Nothing in
+ *     it has to start from zero (every partial that is read has been written by the same call), but two calls
+ *     that overlap on the GPU -- different streams, or different host threads -- race on it.  Issue them on one
+ *     stream, or order them with events. */
+#define AD_STATIC_SCRATCH_BYTES (1u << 20)
+int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d, int32_t vocab,
+                           int32_t* argmax, int32_t* status, void* stream);
+
 /* y [M, N] (FP32) = x [M, K] W^T + bias, W [N, K] in `dtype` (Section 2 projections).  bias may be NULL.
  * BF16 needs K % 64 == 0 and M <= 256. */
 int ad_linear(const void* x, const void* W, const float* bias, int32_t dtype, int32_t M, int32_t K,

@@ -22,6 +22,7 @@ EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
     "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync",
     "ad_debug_logits", "ad_debug_encoder_memory", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
+    "ad_vocab_argmax_static",
     "ad_linear",
 ]
 
@@ -89,6 +90,7 @@ def load():
         "ad_debug_encoder_memory": (C.c_int, [vp, i32, vp, sz]),
         "ad_vocab_argmax_scratch_bytes": (sz, [i32, i32]),
         "ad_vocab_argmax": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, sz, vp, vp]),
+        "ad_vocab_argmax_static": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "ad_linear": (C.c_int, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -328,6 +330,32 @@ def vocab_argmax(x_t, emb_t, status_t=None):
         raise AdError(rc, "ad_vocab_argmax")
     torch.cuda.synchronize()
     return out
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def vocab_argmax_static(x_t, emb_t, out_t, status_t=None):
+    """Projection + arg-max for callers that must not allocate device memory at call time.
+
+    Unlike :func:`vocab_argmax`, nothing is allocated here or inside the library: ``out_t`` (int32, [M]) is
+    the caller's, and the scratch is an array built into the library (1 MiB per GPU).  Problems that need
+    more are refused with ``AD_ERR_CAPACITY``.  Calls on one GPU share that array, so keep them on one
+    stream; make the first call on a device outside any stream capture.  Asynchronous on torch's current
+    stream."""
+    import torch
+    lib = load()
+    M, d = x_t.shape
+    V = emb_t.shape[0]
+    dtype = AD_DTYPE_BF16 if x_t.dtype == torch.bfloat16 else AD_DTYPE_FP32
+    rc = lib.ad_vocab_argmax_static(C.c_void_p(x_t.data_ptr()), C.c_void_p(emb_t.data_ptr()), dtype, M, d, V,
+                                    C.c_void_p(out_t.data_ptr()),
+                                    C.c_void_p(status_t.data_ptr()) if status_t is not None else None,
+                                    C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc != AD_OK:
+        msg = lib.ad_last_error(None)
+        raise AdError(rc, msg.decode() if msg else "ad_vocab_argmax_static")
+    return out_t
 
 
 def linear(x_t, W_t, bias_t=None, status_t=None):

@@ -978,3 +978,34 @@ extern "C" int ad_linear(const void* x, const void* W, const float* bias, int32_
   }
   return e == cudaSuccess ? AD_OK : AD_ERR_CUDA;
 }
+
+// ---- projection + arg-max for callers that cannot allocate -------------------------------------------
+// The scratch that ad_vocab_argmax takes from its caller is, here, a fixed array inside the library image.
+// In host code the array's name is only a handle for the runtime, not a device address: the address is asked
+// for once per device (cudaGetSymbolAddress with that device current) and then passed to the kernels.
+static __device__ __align__(256) unsigned char g_static_scratch[AD_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d,
+                                      int32_t vocab, int32_t* argmax, int32_t* status, void* stream) {
+  if (!x || !emb || !argmax || M < 1 || d < 1 || vocab < 1) return fail(nullptr, AD_ERR_ARG, "ad_vocab_argmax_static: bad argument");
+  const size_t need = ad_vocab_argmax_scratch_bytes(vocab, M);
+  if (need > AD_STATIC_SCRATCH_BYTES)
+    return fail(nullptr, AD_ERR_CAPACITY, "ad_vocab_argmax_static: problem needs " + std::to_string(need) +
+                " bytes of scratch, the built-in array holds " + std::to_string((size_t)AD_STATIC_SCRATCH_BYTES));
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return fail(nullptr, AD_ERR_CUDA, "ad_vocab_argmax_static: no current CUDA device");
+  if (!g_static_scratch_addr[dev]) {   // first call on this device: resolve the array's device address
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p)
+      return fail(nullptr, AD_ERR_CUDA, std::string("ad_vocab_argmax_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+    g_static_scratch_addr[dev] = p;
+  }
+  return ad_vocab_argmax(x, emb, dtype, M, d, vocab, argmax, g_static_scratch_addr[dev], AD_STATIC_SCRATCH_BYTES, status, stream);
+}
