@@ -12,7 +12,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libad_b200.so")
+LIB_PATH = os.environ.get("AD_LIB_PATH", os.path.join(_HERE, "libad_b200.so"))
 
 AD_OK, AD_ERR_ARG, AD_ERR_STATE, AD_ERR_CAPACITY, AD_ERR_TIMEOUT, AD_ERR_CUDA = 0, -1, -2, -3, -4, -5
 AD_DTYPE_FP32, AD_DTYPE_BF16 = 0, 1

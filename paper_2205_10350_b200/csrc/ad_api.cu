@@ -2,6 +2,7 @@
 // replay of the decode loop, and the extern "C" entry points declared in include/aggressive_decoding.h.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -50,7 +51,17 @@ struct PassCfg {
   int M_cap = 0;     // packed-token capacity of this pass kind
   int ntile = 16;    // tokens per GEMM tile
   int seg_max = 0;   // longest segment of one row
+  int max_split = 1; // largest split-K factor this pass may use (sizes the partial-sum buffer)
   PassPlan plan;
+  // Split-K factor of a projection that feeds the LayerNorm kernel: enough CTAs to cover the SMs when the
+  // token dimension alone gives only a handful of tiles (power of two, divides the K blocks, <= max_split).
+  int ksplit_for(int N, int K) const {
+    const int tiles = ((N + 127) / 128) * ((M_cap + ntile - 1) / ntile);
+    const int kb = K / 64;
+    int s = 1;
+    while (s * 2 <= max_split && tiles * s * 2 <= 160 && kb % (s * 2) == 0) s *= 2;
+    return s;
+  }
 };
 
 thread_local std::string g_create_error;
@@ -158,6 +169,7 @@ void plan_take(Bump& bp, PassPlan& pl, int B, int M_cap) {
   pl.seg_off = (int*)bp.take(sizeof(int) * B, 256);
   pl.seg_len = (int*)bp.take(sizeof(int) * B, 256);
   pl.key_base = (int*)bp.take(sizeof(int) * B, 256);
+  pl.row_nk = (int*)bp.take(sizeof(int) * B, 256);
   pl.tok_row = (int*)bp.take(sizeof(int) * M_cap, 256);
   pl.tok_pos = (int*)bp.take(sizeof(int) * M_cap, 256);
   pl.tok_id = (int*)bp.take(sizeof(int) * M_cap, 256);
@@ -174,6 +186,7 @@ void pass_shapes(const ad_model_cfg& c, PassCfg* pass, int* M_all) {
   for (int k = 0; k < PK_COUNT; ++k) {
     pass[k].M_cap = B * pass[k].seg_max;
     pass[k].ntile = clampi(pow2ceil(pass[k].M_cap), 16, 256);
+    pass[k].max_split = pass[k].M_cap <= 256 ? 16 : 1;
     if (pass[k].M_cap > all) all = pass[k].M_cap;
   }
   if (!c.has_drafter) { /* the drafter pass is never run; keep its shapes for sizing simplicity */ }
@@ -189,7 +202,9 @@ size_t layout(ad_handle* h, void* base) {
   const int M_all = h->M_all, Mv = h->pass[PK_VERIFY].M_cap;
   const int M_tmp = std::max(h->pass[PK_DRAFT].M_cap, h->pass[PK_ENCODE].M_cap);
   h->y = (float*)bp.take(sizeof(float) * (size_t)M_all * d);
-  h->pre = (float*)bp.take(sizeof(float) * (size_t)M_all * d);
+  size_t pre_elems = 0;
+  for (int k = 0; k < PK_COUNT; ++k) pre_elems = std::max(pre_elems, (size_t)h->pass[k].max_split * h->pass[k].M_cap * d);
+  h->pre = (float*)bp.take(sizeof(float) * pre_elems);
   h->yb.ptr = bp.take(e * (size_t)M_all * d); h->yb.cols = d;
   h->abuf.ptr = bp.take(e * (size_t)M_all * d); h->abuf.cols = d;
   h->hbuf.ptr = bp.take(e * (size_t)M_all * F); h->hbuf.cols = F;
@@ -236,6 +251,7 @@ int check_cfg(const ad_model_cfg* c, std::string* why) {
   if (c->d_model <= 0 || c->n_heads <= 0 || c->d_model % c->n_heads) return bad("d_model must be a positive multiple of n_heads");
   const int dh = c->d_model / c->n_heads;
   if (dh != 32 && dh != 64) return bad("head dimension must be 32 or 64");
+  if (c->d_model > 1024) return bad("d_model must be at most 1024");
   if (c->d_ffn <= 0 || c->vocab <= 4 || c->n_enc < 1 || c->n_dec < 1) return bad("bad model sizes");
   if (c->dtype != AD_DTYPE_FP32 && c->dtype != AD_DTYPE_BF16) return bad("dtype must be AD_DTYPE_FP32 or AD_DTYPE_BF16");
   if (c->dtype == AD_DTYPE_BF16 && (c->d_model % 64 || c->d_ffn % 64)) return bad("BF16 needs d_model and d_ffn to be multiples of 64");
@@ -287,11 +303,40 @@ int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
 
 // ---- kernel launch helpers -----------------------------------------------------------------------
 
-int tc_stages(int ntile, int K) {
+bool g_use_pdl = true;   // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
+
+// Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
+// themselves wait with griddepcontrol.wait before touching anything a predecessor writes).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_use_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+
+int num_sms() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+// Ring depth: as deep as ~200 KB of shared memory allows when the grid fits one wave; when a small-token GEMM
+// has more CTAs than SMs (the vocabulary projection), half of that so that two CTAs share an SM and the
+// whole grid is resident at once.
+int tc_stages(int ntile, int kb, int n_ctas) {
   const int stage = tc::A_STAGE_BYTES + ntile * tc::BLOCK_K * 2;
-  int s = (200 * 1024) / stage;
-  s = clampi(s, 1, tc::MAX_STAGES);
-  const int kb = K / tc::BLOCK_K;
+  const int budget = (ntile <= 64 && n_ctas > num_sms()) ? 100 * 1024 : 200 * 1024;
+  int s = clampi(budget / stage, 1, tc::MAX_STAGES);
   return s < kb ? s : (kb > 0 ? kb : 1);
 }
 
@@ -303,18 +348,17 @@ cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap&
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int stages = tc_stages(p.ntile, p.K);
+  const int ksplit = (EPI == EPI_F32 && p.ksplit > 1) ? p.ksplit : 1;
+  dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile, ksplit);
+  const int stages = tc_stages(p.ntile, (p.K / tc::BLOCK_K) / ksplit, grid.x * grid.y * grid.z);
   const size_t smem = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2) + 1024;
-  dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile);
-  tc::gemm_tc_kernel<EPI><<<grid, 128, smem, st>>>(mw, mx, p, stages);
-  return cudaGetLastError();
+  return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(128), smem, st, mw, mx, p, stages);
 }
 
 template <int EPI>
 cudaError_t launch_simt(cudaStream_t st, const void* w, const void* x, const GemmParams& p, int M_cap) {
   dim3 grid((p.N + 127) / 128, (M_cap + simt::TOK - 1) / simt::TOK);
-  simt::gemm_f32_kernel<EPI><<<grid, 128, 0, st>>>((const float*)w, (const float*)x, p);
-  return cudaGetLastError();
+  return launch_k(simt::gemm_f32_kernel<EPI>, grid, dim3(128), 0, st, (const float*)w, (const float*)x, p);
 }
 
 int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int* M_ptr, int M_cap, GemmParams p) {
@@ -323,6 +367,7 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   h->launches++;
   if (h->bf16) {
     p.ntile = h->pass[pk].ntile;
+    if (epi != EPI_F32) p.ksplit = 1;
     switch (epi) {
       case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, X.map[pk], p, M_cap); break;
       case EPI_ACT: e = launch_tc<EPI_ACT>(h->stream, W.map, X.map[pk], p, M_cap); break;
@@ -354,37 +399,53 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   const int dh = c.d_model / c.n_heads;
   p.scale = 1.0f / sqrtf((float)dh);
   dim3 grid(h->dims.B * p.qchunks, c.n_heads);
+  const dim3 block(256);
   h->launches++;
+  cudaError_t e;
   if (h->bf16) {
-    if (dh == 64) attention_kernel<bf16, 64><<<grid, 128, 0, h->stream>>>(p);
-    else attention_kernel<bf16, 32><<<grid, 128, 0, h->stream>>>(p);
+    if (dh == 64) e = launch_k(attention_kernel<bf16, 64>, grid, block, 0, h->stream, p);
+    else e = launch_k(attention_kernel<bf16, 32>, grid, block, 0, h->stream, p);
   } else {
-    if (dh == 64) attention_kernel<float, 64><<<grid, 128, 0, h->stream>>>(p);
-    else attention_kernel<float, 32><<<grid, 128, 0, h->stream>>>(p);
+    if (dh == 64) e = launch_k(attention_kernel<float, 64>, grid, block, 0, h->stream, p);
+    else e = launch_k(attention_kernel<float, 32>, grid, block, 0, h->stream, p);
   }
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
   return AD_OK;
 }
 
-int layernorm(ad_handle* h, const PassCfg& pc, const float* g, const float* b) {
+// y = LN(sum of the nsplit partial projections in `pre` + bias + y)
+int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, const float* g, const float* b) {
   const int d = h->cfg.d_model;
-  dim3 grid((pc.M_cap + 3) / 4);
+  dim3 grid(pc.M_cap);
+  const size_t stride = (size_t)pc.M_cap * d;
   h->launches++;
-  if (h->bf16) layernorm_kernel<bf16><<<grid, 128, 0, h->stream>>>(pc.plan.M, h->pre, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
-  else layernorm_kernel<float><<<grid, 128, 0, h->stream>>>(pc.plan.M, h->pre, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e;
+  if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+                            (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
+  else e = launch_k(layernorm_kernel<float>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+                    (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("layernorm launch: ") + cudaGetErrorString(e));
   return AD_OK;
+}
+
+// Projection whose consumer is the residual + LayerNorm kernel: written as split-K partial sums, bias left to
+// the consumer.  Returns the number of partials through *nsplit.
+int gemm_to_ln(ad_handle* h, const Mat& W, const ActBuf& X, int pk, int* nsplit) {
+  PassCfg& pc = h->pass[pk];
+  GemmParams o = {};
+  o.out_f32 = h->pre;
+  o.ksplit = h->bf16 ? pc.ksplit_for(W.N, W.K) : 1;
+  *nsplit = o.ksplit;
+  return gemm(h, EPI_F32, W, X, pk, pc.plan.M, pc.M_cap, o);
 }
 
 int embed(ad_handle* h, const PassCfg& pc, const Model& m) {
   const int d = h->cfg.d_model;
   const float sc = sqrtf((float)d);
   h->launches++;
-  if (h->bf16) embed_kernel<bf16, bf16><<<pc.M_cap, 128, 0, h->stream>>>(pc.plan, (const bf16*)m.emb.ptr, h->pe, d, sc, h->y, (bf16*)h->yb.ptr);
-  else embed_kernel<float, float><<<pc.M_cap, 128, 0, h->stream>>>(pc.plan, (const float*)m.emb.ptr, h->pe, d, sc, h->y, (float*)h->yb.ptr);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e;
+  if (h->bf16) e = launch_k(embed_kernel<bf16, bf16>, dim3(pc.M_cap), dim3(128), 0, h->stream, pc.plan, (const bf16*)m.emb.ptr, (const float*)h->pe, d, sc, h->y, (bf16*)h->yb.ptr);
+  else e = launch_k(embed_kernel<float, float>, dim3(pc.M_cap), dim3(128), 0, h->stream, pc.plan, (const float*)m.emb.ptr, (const float*)h->pe, d, sc, h->y, (float*)h->yb.ptr);
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("embed launch: ") + cudaGetErrorString(e));
   return AD_OK;
 }
@@ -399,11 +460,10 @@ int self_attention_sublayer(ad_handle* h, int pk, const Mat& wqkv, const float* 
   p.bias = bqkv; p.dst[0] = h->qbuf; p.dst[1] = kbuf; p.dst[2] = vbuf; p.seg_width = h->cfg.d_model; p.n_direct = 1;
   p.slot = pc.plan.kv_slot;
   AD_TRY(gemm(h, EPI_SCATTER, wqkv, h->yb, pk, pc.plan.M, pc.M_cap, p));
-  AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, nullptr));
-  GemmParams o = {};
-  o.bias = bo; o.out_f32 = h->pre; o.resid = h->y;
-  AD_TRY(gemm(h, EPI_F32, wo, h->abuf, pk, pc.plan.M, pc.M_cap, o));
-  return layernorm(h, pc, lng, lnb);
+  AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, pc.plan.row_nk));
+  int ns = 1;
+  AD_TRY(gemm_to_ln(h, wo, h->abuf, pk, &ns));
+  return layernorm(h, pc, ns, bo, lng, lnb);
 }
 
 int ffn_sublayer(ad_handle* h, int pk, const Mat& w1, const float* b1, const Mat& w2, const float* b2, const float* lng,
@@ -412,10 +472,9 @@ int ffn_sublayer(ad_handle* h, int pk, const Mat& w1, const float* b1, const Mat
   GemmParams a = {};
   a.bias = b1; a.relu = 1; a.out_act = h->hbuf.ptr;
   AD_TRY(gemm(h, EPI_ACT, w1, h->yb, pk, pc.plan.M, pc.M_cap, a));
-  GemmParams o = {};
-  o.bias = b2; o.out_f32 = h->pre; o.resid = h->y;
-  AD_TRY(gemm(h, EPI_F32, w2, h->hbuf, pk, pc.plan.M, pc.M_cap, o));
-  return layernorm(h, pc, lng, lnb);
+  int ns = 1;
+  AD_TRY(gemm_to_ln(h, w2, h->hbuf, pk, &ns));
+  return layernorm(h, pc, ns, b2, lng, lnb);
 }
 
 // Decoder stack over the packed tokens of pass pk (verification: cached, block-causal; drafter: no cache,
@@ -436,10 +495,9 @@ int decoder_pass(ad_handle* h, int pk, Model& m) {
     AD_TRY(gemm(h, EPI_ACT, L.cq, h->yb, pk, pc.plan.M, pc.M_cap, q));
     AD_TRY(attention(h, pc, h->qbuf, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
                      h->st.cross_base, nullptr, h->st.srclen));
-    GemmParams o = {};
-    o.bias = L.cbo; o.out_f32 = h->pre; o.resid = h->y;
-    AD_TRY(gemm(h, EPI_F32, L.co, h->abuf, pk, pc.plan.M, pc.M_cap, o));
-    AD_TRY(layernorm(h, pc, L.ln2g, L.ln2b));
+    int ns = 1;
+    AD_TRY(gemm_to_ln(h, L.co, h->abuf, pk, &ns));
+    AD_TRY(layernorm(h, pc, ns, L.cbo, L.ln2g, L.ln2b));
     AD_TRY(ffn_sublayer(h, pk, L.w1, L.b1, L.w2, L.b2, L.ln3g, L.ln3b));
   }
   return AD_OK;
@@ -476,18 +534,16 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts) {
   p.part_val = h->part_val; p.part_idx = h->part_idx;
   AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   h->launches++;
-  argmax_accept_kernel<<<h->dims.B, 128, 0, h->stream>>>(h->st, pc.plan, h->dims, h->part_val, h->part_idx, h->n_vtiles,
-                                                       pc.M_cap, to_drafts);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(128), 0, h->stream, h->st, pc.plan, h->dims, h->part_val, h->part_idx, h->n_vtiles,
+                                                       pc.M_cap, to_drafts));
   h->last_vocab_which = to_drafts ? 1 : 0;
   return AD_OK;
 }
 
 int prepare_verify(ad_handle* h, int source, int k_cap, const int* ovr, int ovr_len) {
   h->launches++;
-  prepare_verify_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, source, k_cap, ovr,
-                                                 h->cfg.max_tgt, ovr_len);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(prepare_verify_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, source, k_cap, ovr,
+                                                 h->cfg.max_tgt, ovr_len));
   return AD_OK;
 }
 
@@ -495,15 +551,13 @@ int prepare_verify(ad_handle* h, int source, int k_cap, const int* ovr, int ovr_
 int draft_stage(ad_handle* h, int k_cap) {
   AD_TRY(prepare_verify(h, SRC_SIZES, k_cap, nullptr, 0));
   h->launches++;
-  plan_draft_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->pass[PK_DRAFT].plan, h->dims);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(plan_draft_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->pass[PK_DRAFT].plan, h->dims));
   AD_TRY(decoder_pass(h, PK_DRAFT, h->nar));
   const int d = h->cfg.d_model;
   PassCfg& pv = h->pass[PK_VERIFY];
   h->launches++;
-  if (h->bf16) gather_rows_kernel<bf16><<<pv.M_cap, 128, 0, h->stream>>>(pv.plan.M, h->st.gidx, (const bf16*)h->yb.ptr, (bf16*)h->xg.ptr, d);
-  else gather_rows_kernel<float><<<pv.M_cap, 128, 0, h->stream>>>(pv.plan.M, h->st.gidx, (const float*)h->yb.ptr, (float*)h->xg.ptr, d);
-  AD_CUDA(h, cudaGetLastError());
+  if (h->bf16) AD_CUDA(h, launch_k(gather_rows_kernel<bf16>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const bf16*)h->yb.ptr, (bf16*)h->xg.ptr, d));
+  else AD_CUDA(h, launch_k(gather_rows_kernel<float>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const float*)h->yb.ptr, (float*)h->xg.ptr, d));
   return vocab_stage(h, h->nar, h->xg, 1);
 }
 
@@ -514,8 +568,7 @@ int verify_stage(ad_handle* h) {
 
 int commit_stage(ad_handle* h, const int* n_dev) {
   h->launches++;
-  commit_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, n_dev);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(commit_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, n_dev));
   return AD_OK;
 }
 
@@ -673,8 +726,7 @@ extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, c
   AD_CUDA(h, cudaMemcpy2DAsync(h->st.src, sizeof(int) * c.max_src, src, sizeof(int) * src_stride, sizeof(int) * w, B, to_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, src_len, sizeof(int) * B, to_dev(on_host), h->stream));
   h->launches++;
-  plan_encode_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_ENCODE].plan, h->dims);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(plan_encode_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_ENCODE].plan, h->dims));
   AD_TRY(encoder_pass(h, h->ar, true));
   if (c.has_drafter) AD_TRY(encoder_pass(h, h->nar, false));
   h->encoded = true;
@@ -703,8 +755,7 @@ extern "C" int ad_verify_block(ad_handle* h, const int32_t* drafts, const int32_
     return read_status(h);
   }
   h->launches++;
-  export_block_kernel<<<B, 64, 0, h->stream>>>(h->st, h->dims, argmax, n_accepted, nullptr, nullptr, h->pass[PK_VERIFY].plan);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(export_block_kernel, dim3(B), dim3(64), 0, h->stream, h->st, h->dims, argmax, n_accepted, nullptr, nullptr, h->pass[PK_VERIFY].plan));
   return AD_OK;
 }
 
@@ -728,8 +779,7 @@ extern "C" int ad_force_commit(ad_handle* h, const int32_t* tokens, const int32_
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_drafts, tokens, sizeof(int) * (size_t)h->B * h->cfg.kmax, to_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, n, sizeof(int) * h->B, to_dev(on_host), h->stream));
   h->launches++;
-  force_commit_kernel<<<1, 256, 0, h->stream>>>(h->st, h->pass[PK_VERIFY].plan, h->dims, h->st.user_drafts, h->st.user_n);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(force_commit_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, h->st.user_drafts, h->st.user_n));
   if (on_host) return read_status(h);
   return AD_OK;
 }
@@ -748,8 +798,7 @@ extern "C" int ad_draft_block(ad_handle* h, int32_t k_cap, int32_t* drafts, int3
     return read_status(h);
   }
   h->launches++;
-  export_block_kernel<<<B, 64, 0, h->stream>>>(h->st, h->dims, nullptr, nullptr, drafts, k, h->pass[PK_VERIFY].plan);
-  AD_CUDA(h, cudaGetLastError());
+  AD_CUDA(h, launch_k(export_block_kernel, dim3(B), dim3(64), 0, h->stream, h->st, h->dims, nullptr, nullptr, drafts, k, h->pass[PK_VERIFY].plan));
   return AD_OK;
 }
 
@@ -782,8 +831,7 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
   if (opts->max_len) {
     AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, opts->max_len, sizeof(int) * B, to_dev(on_host), h->stream));
     h->launches++;
-    set_maxlen_kernel<<<(B + 63) / 64, 64, 0, h->stream>>>(h->st, h->dims, h->st.user_n);
-    AD_CUDA(h, cudaGetLastError());
+    AD_CUDA(h, launch_k(set_maxlen_kernel, dim3((B + 63) / 64), dim3(64), 0, h->stream, h->st, h->dims, h->st.user_n));
     if (on_host) {
       max_iters = 1;
       for (int b = 0; b < B; ++b) {
@@ -1009,3 +1057,17 @@ extern "C" int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dt
   }
   return ad_vocab_argmax(x, emb, dtype, M, d, vocab, argmax, g_static_scratch_addr[dev], AD_STATIC_SCRATCH_BYTES, status, stream);
 }
+
+#ifdef AD_TRACE
+// Timeline dump of a tracing build: copies up to cap stamps to the host and optionally clears the buffer.
+extern "C" int ad_debug_trace(unsigned long long* host_buf, int cap, int reset) {
+  unsigned int n = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  if (cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n)) != cudaSuccess) return -1;
+  if (n > (1u << 15)) n = 1u << 15;
+  if ((int)n > cap) n = cap;
+  if (n && cudaMemcpyFromSymbol(host_buf, g_trace_buf, sizeof(unsigned long long) * n) != cudaSuccess) return -1;
+  if (reset) { unsigned int z = 0; cudaMemcpyToSymbol(g_trace_n, &z, sizeof(z)); }
+  return (int)n;
+}
+#endif

@@ -31,6 +31,7 @@ struct PassPlan {
   int* seg_off;    // [B] first packed token of row b
   int* seg_len;    // [B] tokens of row b (0 = row idle)
   int* key_base;   // [B] slot index of self-attention key 0 of row b
+  int* row_nk;     // [B] largest number of self-attention keys any token of row b sees
   int* tok_row;    // [Mmax] batch row of packed token m
   int* tok_pos;    // [Mmax] position fed to the positional table
   int* tok_id;     // [Mmax] input token id
@@ -56,9 +57,9 @@ struct GemmParams {
   int M_cap;             // capacity of the token dimension of the buffers
   const float* bias;     // [N] or null
   int relu;
+  int ksplit;            // EPI_F32 only: blockIdx.z takes K range z/ksplit and writes partial z (1 = no split)
   // EPI_F32
-  float* out_f32;        // [M_cap, N]
-  const float* resid;    // [M_cap, N] or null
+  float* out_f32;        // [ksplit][M_cap, N]: partial sums; the consumer adds them up
   // EPI_ACT
   void* out_act;         // [M_cap, N] float or bf16
   // EPI_SCATTER
@@ -71,6 +72,32 @@ struct GemmParams {
   int* part_idx;         // [n_tiles, M_cap]
   int* status;           // device status word (latches AD_ERR_TIMEOUT), may be null
 };
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start
+// while its predecessor in the stream is still running.  pdl_wait() blocks until the predecessor grid (and,
+// transitively, everything before it) has completed and its writes are visible; everything a kernel does
+// before pdl_wait() must touch only data that no kernel ever writes (weights, the kernel's own shared memory).
+// pdl_launch() lets the successor begin its own pre-wait part.  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Optional timeline tracing (compile with -DAD_TRACE): thread 0 of CTA (0,0,0) of every kernel stamps the
+// global nanosecond timer at entry (phase 0), after the dependency wait (phase 1) and at exit (phase 2).
+#ifdef AD_TRACE
+__device__ unsigned long long g_trace_buf[1 << 15];
+__device__ unsigned int g_trace_n;
+__device__ __forceinline__ void trace_mark(int id, int phase) {
+  if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const unsigned int i = atomicAdd(&g_trace_n, 1u);
+    if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)(id * 4 + phase) << 56);
+  }
+}
+#else
+__device__ __forceinline__ void trace_mark(int, int) {}
+#endif
+enum TraceId { TR_GEMM = 0, TR_ATTN = 8, TR_LN = 9, TR_EMBED = 10, TR_PREPARE = 11, TR_ACCEPT = 12, TR_COMMIT = 13 };
 
 __device__ __forceinline__ void latch_error(int* status, int code) {
   if (status) atomicCAS(status, 0, code);

@@ -23,6 +23,8 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
   __shared__ float red_val[4][TOK];
   __shared__ int red_idx[4][TOK];
 
+  pdl_launch();
+  pdl_wait();
   const int M = p.M_ptr ? *p.M_ptr : p.M_host;
   const int t0 = blockIdx.y * TOK;
   if (t0 >= M) return;
@@ -82,7 +84,13 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
       p.part_idx[(size_t)blockIdx.x * p.M_cap + t0 + tid] = i;
     }
   } else {
-    tc::epilogue_chunk<EPI, float>(p, n, t0, M, acc);
+    __shared__ int slot_s[TOK];
+    if (EPI == EPI_SCATTER) {
+      if (tid < TOK) slot_s[tid] = (t0 + tid < M) ? p.slot[t0 + tid] : 0;
+      __syncthreads();
+    }
+    const float b = (p.bias && n < p.N) ? p.bias[n] : 0.f;
+    tc::epilogue_chunk<EPI, float>(p, n, t0, M, acc, b, p.out_f32, slot_s, 0);
   }
 }
 

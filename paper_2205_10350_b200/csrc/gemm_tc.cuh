@@ -120,30 +120,35 @@ __device__ __forceinline__ void warp_argmax(float& v, int& i) {
 }
 
 // Applies the epilogue to 16 consecutive tokens (m0 .. m0+15) of output feature n held by this thread.
+// b is the bias of feature n (0 when there is none); slot_s holds the K/V slot of every token of the tile.
 template <int EPI, typename ActT>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int n, int m0, int M, const float* acc) {
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int n, int m0, int M, const float* acc, float b,
+                                               float* out_f32, const int* slot_s, int j0) {
   if (n >= p.N) return;
-  const float b = p.bias ? p.bias[n] : 0.f;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     const int m = m0 + j;
     if (m >= M) break;
     float v = acc[j] + b;
     if (EPI == EPI_F32) {
-      if (p.resid) v += p.resid[(size_t)m * p.N + n];
-      p.out_f32[(size_t)m * p.N + n] = v;
+      out_f32[(size_t)m * p.N + n] = v;
     } else if (EPI == EPI_ACT) {
       if (p.relu) v = fmaxf(v, 0.f);
       reinterpret_cast<ActT*>(p.out_act)[(size_t)m * p.N + n] = from_f32<ActT>(v);
     } else if (EPI == EPI_SCATTER) {
       const int s = n / p.seg_width, c = n - s * p.seg_width;
-      const int row = (s < p.n_direct) ? m : p.slot[m];
+      const int row = (s < p.n_direct) ? m : slot_s[j0 + j];
       reinterpret_cast<ActT*>(p.dst[s])[(size_t)row * p.seg_width + c] = from_f32<ActT>(v);
     }
   }
 }
 
-// grid = (ceil(N / 128), ceil(M_cap / ntile)); block = 128 threads; dynamic smem = stages * stage bytes + 1024.
+// grid = (ceil(N / 128), ceil(M_cap / ntile), ksplit); block = 128 threads;
+// dynamic smem = stages * stage bytes + 1024.
+//
+// Order of events in a CTA (the part before pdl_wait() overlaps the previous kernel of the stream):
+//   barriers, TMEM allocation, pdl_launch;  producer: weight tiles of the first ring round (token tile 0 only);
+//   pdl_wait;  token count M;  producer: activation tiles, then the rest of the K loop;  MMA issue;  epilogue.
 template <int EPI>
 __global__ void __launch_bounds__(128, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
@@ -154,24 +159,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __shared__ __align__(8) uint64_t bar_acc;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ float red_val[4][256];
-  __shared__ int red_idx[4][256];
+  __shared__ int slot_s[256];
+  __shared__ float red_val[EPI == EPI_ARGMAX ? 4 : 1][256];
+  __shared__ int red_idx[EPI == EPI_ARGMAX ? 4 : 1][256];
 
-  const int M = p.M_ptr ? *p.M_ptr : p.M_host;
-  const int t0 = blockIdx.y * p.ntile;
-  if (t0 >= M) return;                       // uniform over the CTA: nothing allocated yet
+  trace_mark(TR_GEMM + EPI, 0);
+  const int ntile = p.ntile;
+  const int t0 = blockIdx.y * ntile;
   const int n0 = blockIdx.x * BLOCK_N_FEAT;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ntile = p.ntile;
   const int b_stage_bytes = ntile * BLOCK_K * 2;
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
-  const int num_kb = p.K / BLOCK_K;
+  const int kb_total = p.K / BLOCK_K;
+  const int ksplit = (EPI == EPI_F32 && p.ksplit > 1) ? p.ksplit : 1;
+  const int kb_begin = (int)(((long long)kb_total * blockIdx.z) / ksplit);
+  const int kb_end = (int)(((long long)kb_total * (blockIdx.z + 1)) / ksplit);
+  const int num_kb = kb_end - kb_begin;
+  const int first_round = num_kb < stages ? num_kb : stages;
+  const bool early = (blockIdx.y == 0);   // token tile 0 always has work (M >= 1 whenever a result is read)
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
   uint32_t tmem_cols = 32;
   while (tmem_cols < (uint32_t)ntile) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
@@ -190,84 +203,112 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_base_slot;
+  // Successors may start now: this CTA already owns its tensor memory, so a later kernel's allocation can
+  // never starve it.
+  pdl_launch();
 
-  if (warp == 0 && lane == 0) {
-    // ---- TMA producer ----
-    for (int kb = 0; kb < num_kb; ++kb) {
-      const int s = kb % stages;
-      const uint32_t round = kb / stages;
-      if (round > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (round - 1) & 1, p.status)) { abort_flag = 1; break; }
-      if (*reinterpret_cast<volatile int*>(&abort_flag)) break;
-      const uint32_t a_dst = smem_base + s * stage_bytes;
-      const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-      const uint32_t bar = smem_u32(&bar_full[s]);
+  const bool is_producer = (warp == 0 && lane == 0);
+  if (is_producer && early) {
+    // weights never change: fetch the first ring round before the previous kernel has finished
+    for (int i = 0; i < first_round; ++i) {
+      const uint32_t bar = smem_u32(&bar_full[i]);
       mbar_expect_tx(bar, (uint32_t)stage_bytes);
-      tma_load_2d(a_dst, &map_w, kb * BLOCK_K, n0, bar);
-      tma_load_2d(b_dst, &map_x, kb * BLOCK_K, t0, bar);
+      tma_load_2d(smem_base + i * stage_bytes, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
     }
-  } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer ----
-    const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
-    bool ok = true;
-    for (int kb = 0; kb < num_kb && ok; ++kb) {
-      const int s = kb % stages;
-      const uint32_t round = kb / stages;
-      ok = mbar_wait(smem_u32(&bar_full[s]), round & 1, p.status);
-      if (!ok) { abort_flag = 1; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a_addr = smem_base + s * stage_bytes;
-      const uint64_t desc_a = make_smem_desc(a_addr);
-      const uint64_t desc_b = make_smem_desc(a_addr + A_STAGE_BYTES);
-#pragma unroll
-      for (int k4 = 0; k4 < BLOCK_K / UMMA_K; ++k4) {
-        // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
-        umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-      }
-      umma_commit(smem_u32(&bar_empty[s]));   // stage reusable once these MMAs have read it
-    }
-    if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
   }
-  __syncwarp();
+  const int n = n0 + warp * 32 + lane;
+  const float bias_n = (p.bias && n < p.N) ? p.bias[n] : 0.f;   // a weight as well: no dependency
 
-  // ---- epilogue: all four warps ----
-  bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.status);
-  if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
-  ready = __all_sync(0xffffffffu, ready);
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  if (ready) {
-    const int n = n0 + warp * 32 + lane;
-    for (int c = 0; c < ntile; c += 16) {
-      float acc[16];
-      tmem_ld16(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c), acc);
-      if (EPI == EPI_ARGMAX) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          float v = (n < p.N) ? acc[j] : -INFINITY;
-          int i = n;
-          warp_argmax(v, i);
-          if (lane == 0) { red_val[warp][c + j] = v; red_idx[warp][c + j] = i; }
+  pdl_wait();
+  trace_mark(TR_GEMM + EPI, 1);
+  const int M = p.M_ptr ? *p.M_ptr : p.M_host;
+  const bool valid = early || (t0 < M);
+
+  if (valid) {
+    if (EPI == EPI_SCATTER) {
+      for (int j = threadIdx.x; j < ntile; j += 128) slot_s[j] = (t0 + j < M) ? p.slot[t0 + j] : 0;
+    }
+    if (is_producer) {
+      // ---- TMA producer ----
+      for (int i = 0; i < num_kb; ++i) {
+        const int s = i % stages;
+        const uint32_t round = i / stages;
+        if (round > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (round - 1) & 1, p.status)) { abort_flag = 1; break; }
+        if (*reinterpret_cast<volatile int*>(&abort_flag)) break;
+        const uint32_t a_dst = smem_base + s * stage_bytes;
+        const uint32_t bar = smem_u32(&bar_full[s]);
+        if (!(early && i < first_round)) {
+          mbar_expect_tx(bar, (uint32_t)stage_bytes);
+          tma_load_2d(a_dst, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
         }
-      } else {
-        epilogue_chunk<EPI, bf16>(p, n, t0 + c, M, acc);
+        tma_load_2d(a_dst + A_STAGE_BYTES, &map_x, (kb_begin + i) * BLOCK_K, t0, bar);
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---- MMA issuer ----
+      const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
+      bool ok = true;
+      for (int i = 0; i < num_kb && ok; ++i) {
+        const int s = i % stages;
+        const uint32_t round = i / stages;
+        ok = mbar_wait(smem_u32(&bar_full[s]), round & 1, p.status);
+        if (!ok) { abort_flag = 1; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_base + s * stage_bytes;
+        const uint64_t desc_a = make_smem_desc(a_addr);
+        const uint64_t desc_b = make_smem_desc(a_addr + A_STAGE_BYTES);
+#pragma unroll
+        for (int k4 = 0; k4 < BLOCK_K / UMMA_K; ++k4) {
+          // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
+          umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (i | k4) != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bar_empty[s]));   // stage reusable once these MMAs have read it
+      }
+      if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
+    }
+    __syncwarp();
+
+    // ---- epilogue: all four warps ----
+    bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.status);
+    if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
+    ready = __all_sync(0xffffffffu, ready);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (EPI == EPI_SCATTER) __syncthreads();   // slot_s visible (every thread reaches this point)
+    if (ready) {
+      float* out_f32 = (EPI == EPI_F32) ? p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N : nullptr;
+      for (int c = 0; c < ntile; c += 16) {
+        if (t0 + c >= M) break;
+        float acc[16];
+        tmem_ld16(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c), acc);
+        if (EPI == EPI_ARGMAX) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            float v = (n < p.N) ? acc[j] : -INFINITY;
+            int i = n;
+            warp_argmax(v, i);
+            if (lane == 0) { red_val[warp][c + j] = v; red_idx[warp][c + j] = i; }
+          }
+        } else {
+          epilogue_chunk<EPI, bf16>(p, n, t0 + c, M, acc, bias_n, out_f32, slot_s, c);
+        }
       }
     }
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (EPI == EPI_ARGMAX && ready) {
-    for (int j = threadIdx.x; j < ntile; j += blockDim.x) {
-      const int m = t0 + j;
-      if (m < M) {
-        float v = red_val[0][j];
-        int i = red_idx[0][j];
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (EPI == EPI_ARGMAX && ready) {
+      for (int j = threadIdx.x; j < ntile; j += blockDim.x) {
+        const int m = t0 + j;
+        if (m < M) {
+          float v = red_val[0][j];
+          int i = red_idx[0][j];
 #pragma unroll
-        for (int w = 1; w < 4; ++w) {
-          const float ov = red_val[w][j];
-          const int oi = red_idx[w][j];
-          if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+          for (int w = 1; w < 4; ++w) {
+            const float ov = red_val[w][j];
+            const int oi = red_idx[w][j];
+            if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+          }
+          p.part_val[(size_t)blockIdx.x * p.M_cap + m] = v;
+          p.part_idx[(size_t)blockIdx.x * p.M_cap + m] = i;
         }
-        p.part_val[(size_t)blockIdx.x * p.M_cap + m] = v;
-        p.part_idx[(size_t)blockIdx.x * p.M_cap + m] = i;
       }
     }
   }
@@ -275,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
   }
+  trace_mark(TR_GEMM + EPI, 2);
 }
 
 }  // namespace tc

@@ -80,6 +80,10 @@ __device__ int warp_suffix_match(const int* out, int j, const int* src, int n, i
 __global__ void __launch_bounds__(256)
 prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap, const int* override_stream,
                       int override_stride, int override_len) {
+  trace_mark(TR_PREPARE, 0);
+  pdl_launch();
+  pdl_wait();
+  trace_mark(TR_PREPARE, 1);
   __shared__ int s_k[256];
   __shared__ int s_off[257];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -136,6 +140,7 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
       plan.seg_off[b] = off;
       plan.seg_len[b] = k;
       plan.key_base[b] = b * dm.max_tgt;
+      plan.row_nk[b] = len + k;
     }
     for (int i = lane; i < k; i += 32) {
       if (source == SRC_USER) dr[i] = st.user_drafts[(size_t)b * dm.kmax + i];
@@ -162,6 +167,8 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 plan_draft_kernel(DevState st, PassPlan blk, PassPlan plan, Dims dm) {
+  pdl_launch();
+  pdl_wait();
   __shared__ int s_off[257];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int B = dm.B;
@@ -179,7 +186,7 @@ plan_draft_kernel(DevState st, PassPlan blk, PassPlan plan, Dims dm) {
   for (int b = warp; b < B; b += 8) {
     const int k = blk.seg_len[b], len = st.len[b], off = s_off[b];
     const int n = k > 0 ? len + 1 + k : 0;
-    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; }
+    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; plan.row_nk[b] = n; }
     for (int i = lane; i < n; i += 32) {
       const int m = off + i;
       plan.tok_row[m] = b;
@@ -198,6 +205,8 @@ plan_draft_kernel(DevState st, PassPlan blk, PassPlan plan, Dims dm) {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
+  pdl_launch();
+  pdl_wait();
   __shared__ int s_off[257];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int B = dm.B;
@@ -216,7 +225,7 @@ plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
   __syncthreads();
   for (int b = warp; b < B; b += 8) {
     const int n = st.srclen[b], off = s_off[b];
-    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; }
+    if (lane == 0) { plan.seg_off[b] = off; plan.seg_len[b] = n; plan.key_base[b] = off; plan.row_nk[b] = n; }
     for (int i = lane; i < n; i += 32) {
       const int m = off + i;
       plan.tok_row[m] = b;
@@ -230,6 +239,8 @@ plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
 }
 
 __global__ void set_maxlen_kernel(DevState st, Dims dm, const int* maxlen) {
+  pdl_launch();
+  pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < dm.B) {
     int v = maxlen[b];
@@ -246,6 +257,8 @@ template <typename WT, typename ActT>
 __global__ void __launch_bounds__(128)
 embed_kernel(PassPlan plan, const WT* __restrict__ emb, const float* __restrict__ pe, int d, float scale,
              float* __restrict__ y, ActT* __restrict__ yb) {
+  pdl_launch();
+  pdl_wait();
   const int m = blockIdx.x;
   if (m >= *plan.M) return;
   const int id = plan.tok_id[m], pos = plan.tok_pos[m];
@@ -257,31 +270,100 @@ embed_kernel(PassPlan plan, const WT* __restrict__ emb, const float* __restrict_
 }
 
 // ---------------------------------------------------------------------------------------------
-// LayerNorm (biased variance) of pre[m, :]; one warp per packed token.  grid = ceil(M_cap / 4), block = 128.
+// Residual + LayerNorm:  x = sum_s pre[s][m, :] + bias + resid[m, :];  y = LN(x) (biased variance).
+// pre holds the split-K partial sums of the preceding projection (nsplit <= 16 of them, split_stride floats
+// apart).  One CTA per packed token; each thread owns up to two groups of four consecutive features and issues
+// all of its loads (partials, residual) at once, so the kernel costs one global-memory round trip.
+// y may alias resid.  d % 4 == 0, d <= 1024.  grid = M_cap, block = 128.
 // ---------------------------------------------------------------------------------------------
-template <typename ActT>
-__global__ void __launch_bounds__(128)
-layernorm_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, const float* __restrict__ g,
-                 const float* __restrict__ bta, int d, float eps, float* __restrict__ y, ActT* __restrict__ yb) {
-  const int m = blockIdx.x * 4 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (m >= *M_ptr) return;
-  const float* x = pre + (size_t)m * d;
-  float s = 0.f;
-  for (int i = lane; i < d; i += 32) s += x[i];
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-  const float mean = s / (float)d;
-  float v = 0.f;
-  for (int i = lane; i < d; i += 32) { const float t = x[i] - mean; v = fmaf(t, t, v); }
+__device__ __forceinline__ float block_sum_128(float v, float* red) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  const float inv = rsqrtf(v / (float)d + eps);
-  for (int i = lane; i < d; i += 32) {
-    const float o = g[i] * ((x[i] - mean) * inv) + bta[i];
-    y[(size_t)m * d + i] = o;
-    yb[(size_t)m * d + i] = from_f32<ActT>(o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __syncthreads();                 // red may still be read from a previous call
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  return red[0] + red[1] + red[2] + red[3];
+}
+
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void store4(bf16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<unsigned int*>(&a);
+  u.y = *reinterpret_cast<unsigned int*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+template <typename ActT>
+__global__ void __launch_bounds__(128)
+layernorm_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, int nsplit, size_t split_stride,
+                 const float* __restrict__ bias, const float* resid, const float* __restrict__ g,
+                 const float* __restrict__ bta, int d, float eps, float* y, ActT* __restrict__ yb) {
+  __shared__ float red[4];
+  trace_mark(TR_LN, 0);
+  pdl_launch();
+  const int groups = d >> 2;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  // gains and biases are weights: fetch them while the previous kernel is still running
+  float4 gv[2], bv[2], cb[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int gi = threadIdx.x + 128 * i;
+    const bool on = gi < groups;
+    gv[i] = on ? reinterpret_cast<const float4*>(g)[gi] : zero4;
+    bv[i] = on ? reinterpret_cast<const float4*>(bta)[gi] : zero4;
+    cb[i] = (on && bias) ? reinterpret_cast<const float4*>(bias)[gi] : zero4;
   }
+  pdl_wait();
+  trace_mark(TR_LN, 1);
+  const int m = blockIdx.x;
+  if (m >= *M_ptr) return;
+  float4 xv[2];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int gi = threadIdx.x + 128 * i;
+    float4 v = zero4;
+    if (gi < groups) {
+      const size_t off = (size_t)m * groups + gi;
+      float4 part[16];
+#pragma unroll
+      for (int sp = 0; sp < 16; ++sp)
+        part[sp] = (sp < nsplit) ? reinterpret_cast<const float4*>(pre + sp * split_stride)[off] : zero4;
+      const float4 r = resid ? reinterpret_cast<const float4*>(resid)[off] : zero4;
+      v = make_float4(cb[i].x + r.x, cb[i].y + r.y, cb[i].z + r.z, cb[i].w + r.w);
+#pragma unroll
+      for (int sp = 0; sp < 16; ++sp) { v.x += part[sp].x; v.y += part[sp].y; v.z += part[sp].z; v.w += part[sp].w; }
+    }
+    xv[i] = v;
+    s += v.x + v.y + v.z + v.w;
+  }
+  const float mean = block_sum_128(s, red) / (float)d;
+  float vs = 0.f;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    if (threadIdx.x + 128 * i < groups) {
+      const float a = xv[i].x - mean, b = xv[i].y - mean, c = xv[i].z - mean, e = xv[i].w - mean;
+      vs += a * a + b * b + c * c + e * e;
+    }
+  }
+  const float inv = rsqrtf(block_sum_128(vs, red) / (float)d + eps);
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int gi = threadIdx.x + 128 * i;
+    if (gi < groups) {
+      float4 o;
+      o.x = gv[i].x * ((xv[i].x - mean) * inv) + bv[i].x;
+      o.y = gv[i].y * ((xv[i].y - mean) * inv) + bv[i].y;
+      o.z = gv[i].z * ((xv[i].z - mean) * inv) + bv[i].z;
+      o.w = gv[i].w * ((xv[i].w - mean) * inv) + bv[i].w;
+      const size_t off = ((size_t)m * groups + gi) * 4;
+      store4(y + off, o);
+      store4(yb + off, o);
+    }
+  }
+  trace_mark(TR_LN, 2);
 }
 
 // dst[j, :] = src[gidx[j], :] for j < *M_ptr.  grid = M_cap, block = 128.
@@ -289,6 +371,8 @@ template <typename ActT>
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(const int* __restrict__ M_ptr, const int* __restrict__ gidx, const ActT* __restrict__ src,
                    ActT* __restrict__ dst, int d) {
+  pdl_launch();
+  pdl_wait();
   const int j = blockIdx.x;
   if (j >= *M_ptr) return;
   const int s = gidx[j];
@@ -306,6 +390,8 @@ gather_rows_kernel(const int* __restrict__ M_ptr, const int* __restrict__ gidx, 
 __global__ void __launch_bounds__(128)
 argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
                      const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts) {
+  pdl_launch();
+  pdl_wait();
   const int b = blockIdx.x;
   const int k = blk.seg_len[b];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -361,6 +447,8 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
+  pdl_launch();
+  pdl_wait();
   __shared__ int s_active, s_allfin;
   if (threadIdx.x == 0) { s_active = 0; s_allfin = 1; }
   __syncthreads();
@@ -405,6 +493,8 @@ commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
 // Teacher-forced commit: the caller supplies the accepted tokens.  grid = 1, block = 256.
 __global__ void __launch_bounds__(256)
 force_commit_kernel(DevState st, PassPlan blk, Dims dm, const int* tokens, const int* n_in) {
+  pdl_launch();
+  pdl_wait();
   for (int b = threadIdx.x; b < dm.B; b += 256) {
     const int n = n_in[b], k = blk.seg_len[b];
     const int* tk = tokens + (size_t)b * dm.kmax;
@@ -428,6 +518,8 @@ force_commit_kernel(DevState st, PassPlan blk, Dims dm, const int* tokens, const
 // Copies the block results to caller-visible arrays (device pointers).  grid = B, block = 64.
 __global__ void export_block_kernel(DevState st, Dims dm, int* argmax_out, int* n_out, int* drafts_out, int* k_out,
                                     PassPlan blk) {
+  pdl_launch();
+  pdl_wait();
   const int b = blockIdx.x;
   if (argmax_out)
     for (int i = threadIdx.x; i < dm.kmax; i += blockDim.x) argmax_out[(size_t)b * dm.kmax + i] = st.pred[(size_t)b * dm.kmax + i];
@@ -442,6 +534,8 @@ __global__ void export_block_kernel(DevState st, Dims dm, int* argmax_out, int* 
 // FP32 copy of an activation buffer (debug).  grid-stride.
 template <typename ActT>
 __global__ void to_f32_kernel(const ActT* __restrict__ src, float* __restrict__ dst, size_t n) {
+  pdl_launch();
+  pdl_wait();
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = to_f32(src[i]);
 }
