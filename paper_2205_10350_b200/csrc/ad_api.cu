@@ -528,14 +528,14 @@ int encoder_pass(ad_handle* h, Model& m, bool keep_memory) {
 
 // Output projection fused with arg-max over X (yb for the verifier, the gathered mask rows for the drafter),
 // then the final reduction and (verifier) the draft compare.
-int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts) {
+int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto_commit) {
   PassCfg& pc = h->pass[PK_VERIFY];
   GemmParams p = {};
   p.part_val = h->part_val; p.part_idx = h->part_idx;
   AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   h->launches++;
-  AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(128), 0, h->stream, h->st, pc.plan, h->dims, h->part_val, h->part_idx, h->n_vtiles,
-                                                       pc.M_cap, to_drafts));
+  AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
+                      pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1)));
   h->last_vocab_which = to_drafts ? 1 : 0;
   return AD_OK;
 }
@@ -558,12 +558,12 @@ int draft_stage(ad_handle* h, int k_cap) {
   h->launches++;
   if (h->bf16) AD_CUDA(h, launch_k(gather_rows_kernel<bf16>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const bf16*)h->yb.ptr, (bf16*)h->xg.ptr, d));
   else AD_CUDA(h, launch_k(gather_rows_kernel<float>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const float*)h->yb.ptr, (float*)h->xg.ptr, d));
-  return vocab_stage(h, h->nar, h->xg, 1);
+  return vocab_stage(h, h->nar, h->xg, 1, 0);
 }
 
-int verify_stage(ad_handle* h) {
+int verify_stage(ad_handle* h, int auto_commit) {
   AD_TRY(decoder_pass(h, PK_VERIFY, h->ar));
-  return vocab_stage(h, h->ar, h->yb, 0);
+  return vocab_stage(h, h->ar, h->yb, 0, auto_commit);
 }
 
 int commit_stage(ad_handle* h, const int* n_dev) {
@@ -584,8 +584,7 @@ int loop_iteration(ad_handle* h, const ad_gen_opts& o, const int* ovr, int ovr_l
   } else {
     AD_TRY(prepare_verify(h, ovr ? SRC_OVERRIDE : SRC_POLICY, o.k, ovr, ovr_len));
   }
-  AD_TRY(verify_stage(h));
-  return commit_stage(h, nullptr);
+  return verify_stage(h, 1);   // accept and commit in one kernel
 }
 
 int read_status(ad_handle* h) {
@@ -748,7 +747,7 @@ extern "C" int ad_verify_block(ad_handle* h, const int32_t* drafts, const int32_
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_drafts, drafts, sizeof(int) * (size_t)B * c.kmax, to_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_k, k, sizeof(int) * B, to_dev(on_host), h->stream));
   AD_TRY(prepare_verify(h, SRC_USER, c.kmax, nullptr, 0));
-  AD_TRY(verify_stage(h));
+  AD_TRY(verify_stage(h, 0));
   if (on_host) {
     if (argmax) AD_CUDA(h, cudaMemcpyAsync(argmax, h->st.pred, sizeof(int) * (size_t)B * c.kmax, cudaMemcpyDeviceToHost, h->stream));
     if (n_accepted) AD_CUDA(h, cudaMemcpyAsync(n_accepted, h->st.n_acc, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));

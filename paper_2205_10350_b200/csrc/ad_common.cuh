@@ -82,7 +82,8 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Optional timeline tracing (compile with -DAD_TRACE): thread 0 of CTA (0,0,0) of every kernel stamps the
-// global nanosecond timer at entry (phase 0), after the dependency wait (phase 1) and at exit (phase 2).
+// global nanosecond timer at entry (phase 0), after the dependency wait (phase 1), at exit (phase 2) and at
+// kernel-specific points in between (phases 3..7).
 #ifdef AD_TRACE
 __device__ unsigned long long g_trace_buf[1 << 15];
 __device__ unsigned int g_trace_n;
@@ -91,7 +92,7 @@ __device__ __forceinline__ void trace_mark(int id, int phase) {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     const unsigned int i = atomicAdd(&g_trace_n, 1u);
-    if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)(id * 4 + phase) << 56);
+    if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)(id * 8 + phase) << 56);
   }
 }
 #else

@@ -96,6 +96,22 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
+// 32 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
@@ -107,6 +123,23 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Order-preserving map from float to unsigned: a > b  <=>  key(a) > key(b) (no NaNs expected).
+__device__ __forceinline__ unsigned int float_key(float v) {
+  const unsigned int u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(unsigned int k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+// Largest value over the warp and the lowest lane holding it: one redux and one ballot.
+__device__ __forceinline__ void warp_argmax_lane(float v, float& best, int& lane_of_best) {
+  const unsigned int k = float_key(v);
+  const unsigned int m = __reduce_max_sync(0xffffffffu, k);
+  const unsigned int bal = __ballot_sync(0xffffffffu, k == m);
+  best = key_float(m);
+  lane_of_best = __ffs(bal) - 1;
 }
 
 // Best (value, lowest index) over the 32 lanes of a warp.
@@ -207,10 +240,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   // never starve it.
   pdl_launch();
 
-  const bool is_producer = (warp == 0 && lane == 0);
-  if (is_producer && early) {
+  // TMA issue is spread over lane 0 of all four warps: one thread's bulk-tensor copies are processed one after
+  // the other, several threads' copies run side by side.  Stage i of the first ring round belongs to warp i % 4;
+  // later rounds are fed by warps 0, 2 and 3 (warp 1's lane 0 is busy issuing MMAs).
+  if (early && lane == 0) {
     // weights never change: fetch the first ring round before the previous kernel has finished
-    for (int i = 0; i < first_round; ++i) {
+    for (int i = warp; i < first_round; i += 4) {
       const uint32_t bar = smem_u32(&bar_full[i]);
       mbar_expect_tx(bar, (uint32_t)stage_bytes);
       tma_load_2d(smem_base + i * stage_bytes, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
@@ -221,6 +256,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   pdl_wait();
   trace_mark(TR_GEMM + EPI, 1);
+  if (early && lane == 0) {
+    // activations of the first ring round (the activation buffer is always valid memory; rows beyond M are
+    // simply never stored), issued before the token count is known
+    for (int i = warp; i < first_round; i += 4)
+      tma_load_2d(smem_base + i * stage_bytes + A_STAGE_BYTES, &map_x, (kb_begin + i) * BLOCK_K, t0,
+                  smem_u32(&bar_full[i]));
+  }
   const int M = p.M_ptr ? *p.M_ptr : p.M_host;
   const bool valid = early || (t0 < M);
 
@@ -228,21 +270,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (EPI == EPI_SCATTER) {
       for (int j = threadIdx.x; j < ntile; j += 128) slot_s[j] = (t0 + j < M) ? p.slot[t0 + j] : 0;
     }
-    if (is_producer) {
-      // ---- TMA producer ----
-      for (int i = 0; i < num_kb; ++i) {
+    if (lane == 0 && warp != 1) {
+      // ---- TMA producers: everything that was not issued above ----
+      const int pw = warp == 0 ? 0 : warp - 1;          // 0, 1, 2
+      const int begin = early ? first_round : 0;
+      for (int i = begin + pw; i < num_kb; i += 3) {
         const int s = i % stages;
         const uint32_t round = i / stages;
         if (round > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (round - 1) & 1, p.status)) { abort_flag = 1; break; }
         if (*reinterpret_cast<volatile int*>(&abort_flag)) break;
         const uint32_t a_dst = smem_base + s * stage_bytes;
         const uint32_t bar = smem_u32(&bar_full[s]);
-        if (!(early && i < first_round)) {
-          mbar_expect_tx(bar, (uint32_t)stage_bytes);
-          tma_load_2d(a_dst, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
-        }
+        mbar_expect_tx(bar, (uint32_t)stage_bytes);
+        tma_load_2d(a_dst, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
         tma_load_2d(a_dst + A_STAGE_BYTES, &map_x, (kb_begin + i) * BLOCK_K, t0, bar);
       }
+      if (warp == 0) trace_mark(TR_GEMM + EPI, 3);
     } else if (warp == 1 && lane == 0) {
       // ---- MMA issuer ----
       const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
@@ -261,7 +304,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
           umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (i | k4) != 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bar_empty[s]));   // stage reusable once these MMAs have read it
+        // the stage is handed back to the producers only if a later K block will land in it
+        if (i + stages < num_kb) umma_commit(smem_u32(&bar_empty[s]));
       }
       if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
     }
@@ -272,26 +316,39 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
     ready = __all_sync(0xffffffffu, ready);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    trace_mark(TR_GEMM + EPI, 4);
     if (EPI == EPI_SCATTER) __syncthreads();   // slot_s visible (every thread reaches this point)
     if (ready) {
       float* out_f32 = (EPI == EPI_F32) ? p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N : nullptr;
-      for (int c = 0; c < ntile; c += 16) {
+      for (int c = 0; c < ntile; c += 32) {
         if (t0 + c >= M) break;
-        float acc[16];
-        tmem_ld16(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c), acc);
+        float acc[32];
+        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c);
+        if (ntile - c >= 32) {
+          tmem_ld32(taddr, acc);
+        } else {          // ntile == 16
+          tmem_ld16(taddr, acc);
+#pragma unroll
+          for (int j = 16; j < 32; ++j) acc[j] = 0.f;
+        }
         if (EPI == EPI_ARGMAX) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float v = (n < p.N) ? acc[j] : -INFINITY;
-            int i = n;
-            warp_argmax(v, i);
-            if (lane == 0) { red_val[warp][c + j] = v; red_idx[warp][c + j] = i; }
+          for (int j = 0; j < 32; ++j) {
+            if (c + j < ntile && t0 + c + j < M) {      // uniform over the warp
+              // features grow with the lane, so the lowest winning lane is the lowest winning id
+              float best;
+              int wl;
+              warp_argmax_lane((n < p.N) ? acc[j] : -INFINITY, best, wl);
+              if (lane == 0) { red_val[warp][c + j] = best; red_idx[warp][c + j] = n0 + warp * 32 + wl; }
+            }
           }
         } else {
           epilogue_chunk<EPI, bf16>(p, n, t0 + c, M, acc, bias_n, out_f32, slot_s, c);
+          if (ntile - c >= 32) epilogue_chunk<EPI, bf16>(p, n, t0 + c + 16, M, acc + 16, bias_n, out_f32, slot_s, c + 16);
         }
       }
     }
+    trace_mark(TR_GEMM + EPI, 5);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (EPI == EPI_ARGMAX && ready) {

@@ -257,8 +257,10 @@ template <typename WT, typename ActT>
 __global__ void __launch_bounds__(128)
 embed_kernel(PassPlan plan, const WT* __restrict__ emb, const float* __restrict__ pe, int d, float scale,
              float* __restrict__ y, ActT* __restrict__ yb) {
+  trace_mark(TR_EMBED, 0);
   pdl_launch();
   pdl_wait();
+  trace_mark(TR_EMBED, 1);
   const int m = blockIdx.x;
   if (m >= *plan.M) return;
   const int id = plan.tok_id[m], pos = plan.tok_pos[m];
@@ -380,114 +382,160 @@ gather_rows_kernel(const int* __restrict__ M_ptr, const int* __restrict__ gidx, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Commit of one row (Algorithm 1 lines 6-7): n > 0 appends pred[0..n) to the row's output, advances the cache
+// length, sets the last token and the finished flag; n < 0 rolls |n| committed tokens back; n = 0 discards
+// the block.  Executed by one warp.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void commit_row(const DevState& st, const PassPlan& blk, const Dims& dm, int b, int n,
+                                           int nacc, int lane) {
+  int len = st.len[b];
+  if (n > nacc || (n < 0 && -n > len)) {
+    if (lane == 0) latch_error(st.status, AD_ERR_ARG);
+    n = 0;
+  }
+  __syncwarp();
+  if (n > 0) {
+    const int* pred = st.pred + (size_t)b * dm.kmax;
+    int* out = st.out_ids + (size_t)b * dm.max_tgt;
+    for (int i = lane; i < n; i += 32) out[len + i] = pred[i];
+    if (lane == 0) {
+      const int last = pred[n - 1];
+      len += n;
+      st.len[b] = len;
+      st.last[b] = last;
+      if (last == dm.eos || len >= st.maxlen[b]) st.fin[b] = 1;
+      st.stat_acc[b] += n;
+    }
+  } else if (n < 0 && lane == 0) {
+    len += n;
+    st.len[b] = len;
+    st.last[b] = len > 0 ? st.out_ids[(size_t)b * dm.max_tgt + len - 1] : dm.bos;
+    st.fin[b] = 0;
+  }
+  if (lane == 0) {
+    if (nacc > 0) {
+      st.stat_it[b] += 1;
+      st.stat_off[b] += blk.seg_len[b];
+    }
+    st.n_acc[b] = 0;
+  }
+}
+
+// After every row has been committed: loop counter and the "all rows finished" word.  One thread.
+__device__ __forceinline__ void finish_iteration(const DevState& st, const Dims& dm, bool any_active) {
+  int all = 1;
+  for (int b = 0; b < dm.B; ++b) all &= (__ldcg(st.fin + b) != 0);
+  if (any_active) *st.loop_it += 1;
+  *st.all_fin = all;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Final arg-max over the per-tile partials of the fused projection, then the draft compare:
 //   c = first block position whose greedy choice differs from the draft (Section 3.1.1; definition of c
 //   in Section 3.2), n = c + 1 (the bifurcation token is kept), n = k when nothing differs, cut at the
-//   first accepted [EOS].  One CTA per row; warp 0 takes the decision with ballots.
+//   first accepted [EOS].  One CTA per row, one warp per block position for the reduction; warp 0 takes the
+//   decision with ballots.
 // to_drafts != 0: drafter mode, the choices are written as the row's drafts and nothing is compared.
-// grid = B, block = 128.
+// auto_commit != 0: the row's n_accepted is committed right away (decode loop); the last CTA to finish
+//   updates the loop counter and the all-finished word (done_ctr: rows done in the low half, active rows in
+//   the high half; left at zero).
+// grid = B, block = 1024.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(1024)
 argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
-                     const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts) {
+                     const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts, int auto_commit,
+                     unsigned int* done_ctr) {
+  trace_mark(TR_ACCEPT, 0);
   pdl_launch();
   pdl_wait();
+  trace_mark(TR_ACCEPT, 1);
   const int b = blockIdx.x;
   const int k = blk.seg_len[b];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int* pred = (to_drafts ? st.drafts : st.pred) + (size_t)b * dm.kmax;
-  if (k == 0) {
-    if (tid == 0 && !to_drafts) st.n_acc[b] = 0;
-    return;
-  }
-  const int off = blk.seg_off[b];
-  for (int i = warp; i < k; i += 4) {
-    const int m = off + i;
-    float v = -INFINITY;
-    int idx = 0x7fffffff;
-    for (int t = lane; t < n_tiles; t += 32) {
-      const float ov = part_val[(size_t)t * M_cap + m];
-      const int oi = part_idx[(size_t)t * M_cap + m];
-      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-    }
+  if (k > 0) {
+    const int off = blk.seg_off[b];
+    for (int i = warp; i < k; i += 32) {
+      const int m = off + i;
+      float v = -INFINITY;
+      int idx = 0x7fffffff;
+      for (int t = lane; t < n_tiles; t += 32) {
+        const float ov = part_val[(size_t)t * M_cap + m];
+        const int oi = part_idx[(size_t)t * M_cap + m];
+        if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+      }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+      }
+      if (lane == 0) pred[i] = idx;
     }
-    if (lane == 0) pred[i] = idx;
   }
   if (to_drafts) return;
   __syncthreads();
   if (warp == 0) {
-    const int* dr = st.drafts + (size_t)b * dm.kmax;
-    int n = k;
-    bool found = false;
-    for (int i0 = 0; i0 < k && !found; i0 += 32) {
-      const int i = i0 + lane;
-      const bool mism = (i < k) && (dr[i] < 0 || pred[i] != dr[i]);
-      const unsigned bal = __ballot_sync(0xffffffffu, mism);
-      if (bal) { n = i0 + __ffs(bal); found = true; }
-    }
-    found = false;
-    for (int i0 = 0; i0 < n && !found; i0 += 32) {
-      const int i = i0 + lane;
-      const bool is_eos = (i < n) && (pred[i] == dm.eos);
-      const unsigned bal = __ballot_sync(0xffffffffu, is_eos);
-      if (bal) { n = i0 + __ffs(bal); found = true; }
+    int n = 0;
+    if (k > 0) {
+      const int* dr = st.drafts + (size_t)b * dm.kmax;
+      n = k;
+      bool found = false;
+      for (int i0 = 0; i0 < k && !found; i0 += 32) {
+        const int i = i0 + lane;
+        const bool mism = (i < k) && (dr[i] < 0 || pred[i] != dr[i]);
+        const unsigned bal = __ballot_sync(0xffffffffu, mism);
+        if (bal) { n = i0 + __ffs(bal); found = true; }
+      }
+      found = false;
+      for (int i0 = 0; i0 < n && !found; i0 += 32) {
+        const int i = i0 + lane;
+        const bool is_eos = (i < n) && (pred[i] == dm.eos);
+        const unsigned bal = __ballot_sync(0xffffffffu, is_eos);
+        if (bal) { n = i0 + __ffs(bal); found = true; }
+      }
     }
     if (lane == 0) st.n_acc[b] = n;
+    if (auto_commit) {
+      __syncwarp();
+      commit_row(st, blk, dm, b, n, n, lane);
+      if (lane == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(done_ctr, n > 0 ? 0x10001u : 1u);
+        if ((t & 0xffffu) == (unsigned)dm.B - 1) {
+          __threadfence();
+          finish_iteration(st, dm, ((t >> 16) + (n > 0 ? 1u : 0u)) != 0);
+          *done_ctr = 0;
+        }
+      }
+    }
   }
+  trace_mark(TR_ACCEPT, 2);
 }
 
 // ---------------------------------------------------------------------------------------------
-// Commit: cache-length advance or rollback (Algorithm 1 lines 6-7).  n_in == null commits n_acc.
-// grid = 1, block = 256.
+// Commit as a call of its own (ad_commit): cache-length advance or rollback.  n_in == null commits n_acc.
+// grid = 1, block = 256 (one warp per row at a time).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
+  __shared__ int s_active;
+  trace_mark(TR_COMMIT, 0);
   pdl_launch();
   pdl_wait();
-  __shared__ int s_active, s_allfin;
-  if (threadIdx.x == 0) { s_active = 0; s_allfin = 1; }
+  trace_mark(TR_COMMIT, 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) s_active = 0;
   __syncthreads();
-  for (int b = threadIdx.x; b < dm.B; b += 256) {
+  for (int b = warp; b < dm.B; b += 8) {
     const int nacc = st.n_acc[b];
-    int n = n_in ? n_in[b] : nacc;
-    int len = st.len[b];
-    if (n > nacc || (n < 0 && -n > len)) {
-      latch_error(st.status, AD_ERR_ARG);
-      n = 0;
-    }
-    if (n > 0) {
-      const int* pred = st.pred + (size_t)b * dm.kmax;
-      int* out = st.out_ids + (size_t)b * dm.max_tgt;
-      for (int i = 0; i < n; ++i) out[len + i] = pred[i];
-      len += n;
-      st.len[b] = len;
-      st.last[b] = pred[n - 1];
-      if (pred[n - 1] == dm.eos || len >= st.maxlen[b]) st.fin[b] = 1;
-      st.stat_acc[b] += n;
-    } else if (n < 0) {
-      len += n;
-      st.len[b] = len;
-      st.last[b] = len > 0 ? st.out_ids[(size_t)b * dm.max_tgt + len - 1] : dm.bos;
-      st.fin[b] = 0;
-    }
-    if (nacc > 0) {
-      st.stat_it[b] += 1;
-      st.stat_off[b] += blk.seg_len[b];
-      atomicOr(&s_active, 1);
-    }
-    st.n_acc[b] = 0;
-    if (!st.fin[b]) atomicAnd(&s_allfin, 0);
+    const int n = n_in ? n_in[b] : nacc;
+    __syncwarp();
+    commit_row(st, blk, dm, b, n, nacc, lane);
+    if (lane == 0 && nacc > 0) atomicOr(&s_active, 1);
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    if (s_active) *st.loop_it += 1;
-    *st.all_fin = s_allfin;
-  }
+  if (threadIdx.x == 0) finish_iteration(st, dm, s_active != 0);
 }
 
 // Teacher-forced commit: the caller supplies the accepted tokens.  grid = 1, block = 256.
