@@ -36,6 +36,12 @@ WL = synth.WORKLOADS[2]
 N_SENT = WL.n_batches
 KMAX = 40                      # outputs are at most 40 tokens, so the block cap of 64 never binds
 METRIC, UNIT = "verified_tokens_per_s", "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the projection kernel at this exact shape
+# (profiles/vocab_argmax_gemm_base_M40_ncu_full.txt); set to None whenever that kernel changes.
+NCU_TRAFFIC_BYTES = 32849664
+WORKLOAD_DESC = ("transformer-base (6+6, d512, h8, ffn2048, vocab 32000, bf16) GEC-shaped input-guided decoding, batch 1, "
+                 "source length U[12,40], drafts = own greedy output with 10% of tokens replaced, block = remaining "
+                 "length (cap 64 never binds)")
 
 
 def peaks():
@@ -52,6 +58,19 @@ def sentence_inputs(rank):
         a, b = synth.make_sources(WL, rank * N_SENT + s)
         srcs.append(a[0]); lens.append(int(b[0]))
     return np.stack(srcs).astype(np.int32), np.array(lens, np.int32)
+
+
+def reduce_max_sum(dist, dev, seconds_or_ms, count):
+    """Whole-job figures from per-rank ones: the slowest rank's time and the total unit count.
+    dist is torch.distributed (already initialised) or None for a single process."""
+    if dist is None:
+        return float(seconds_or_ms), int(count)
+    import torch
+    t = torch.tensor([float(seconds_or_ms)], dtype=torch.float64, device=dev)
+    n = torch.tensor([int(count)], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
 
 
 class ClockSampler:
@@ -132,8 +151,7 @@ def run_reference(args, rank, world):
     line = dict(metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * tot_t / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f32", data="synthetic", impl="reference",
-                config=dict(workload="transformer-base GEC-shaped input-guided decoding, batch 1, 90% draft agreement",
-                            sample=base["sample"]),
+                config=dict(workload=WORKLOAD_DESC, sentences_per_step=N_SENT, sample=base["sample"]),
                 cpu_baseline=dict(value=v, unit=UNIT, cores=base["cores"], kind="oracle", sample=base["sample"]),
                 e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line), flush=True)
@@ -219,9 +237,7 @@ def run_ours(args, rank, world, local_rank):
     clocks = sampler.stop()
     t_ms = sum(a.elapsed_time(b) for a, b in ev)
     tokens = agg["accepted"]
-    if dist is not None:
-        tt = torch.tensor([t_ms], device=dev); dist.all_reduce(tt, op=dist.ReduceOp.MAX); t_ms = float(tt.item())
-        tk = torch.tensor([tokens], device=dev, dtype=torch.int64); dist.all_reduce(tk, op=dist.ReduceOp.SUM); tokens = int(tk.item())
+    t_ms, tokens = reduce_max_sum(dist, dev, t_ms, tokens)
     value = tokens / (t_ms * 1e-3)
 
     # end-to-end arm: host buffers through the same C-ABI call, copies inside the timed region (wall clock)
@@ -234,9 +250,7 @@ def run_ours(args, rank, world, local_rank):
         e2e_tok += step_host()
     barrier()
     e2e_t = time.perf_counter() - t0
-    if dist is not None:
-        tt = torch.tensor([e2e_t], device=dev); dist.all_reduce(tt, op=dist.ReduceOp.MAX); e2e_t = float(tt.item())
-        tk = torch.tensor([e2e_tok], device=dev, dtype=torch.int64); dist.all_reduce(tk, op=dist.ReduceOp.SUM); e2e_tok = int(tk.item())
+    e2e_t, e2e_tok = reduce_max_sum(dist, dev, e2e_t, e2e_tok)
     h2d = int(src.nbytes + lens.nbytes + max_len.nbytes + streams.nbytes)
     d2h = int(N_SENT * KMAX * 4 + N_SENT * 4 + N_SENT * (16 + 4 + 4))     # outputs, lengths, statistics and status words
 
@@ -274,7 +288,7 @@ def run_ours(args, rank, world, local_rank):
     t_cold, t_warm = time_vocab(True), time_vocab(False)
     ach = alg_bytes / (t_cold * 1e-3) / 1e9
     roofline = dict(bound="hbm", kernel="gemm_tc_kernel<EPI_ARGMAX> + arg-max reduction (projection fused with row arg-max)",
-                    achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=None,
+                    achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES,
                     peak_source=pk["source"], us_per_launch_cold=t_cold * 1e3, us_per_launch_l2_warm=t_warm * 1e3,
                     algorithmic_bytes=alg_bytes, timing="separate pass after the timed steps, same process and launch shape "
                     "(250 CTAs x 128 threads, 64-token tile); cold = 256 MB L2 flush before each launch")
@@ -294,9 +308,7 @@ def run_ours(args, rank, world, local_rank):
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=t_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                     data="synthetic",
-                    config=dict(workload="transformer-base (6+6, d512, h8, ffn2048, vocab 32000, bf16) GEC-shaped input-guided "
-                                         "decoding, batch 1, source length U[12,40], drafts = own greedy output with 10% of tokens "
-                                         "replaced, block = remaining length (cap 64 never binds)",
+                    config=dict(workload=WORKLOAD_DESC,
                                 sentences_per_step=N_SENT, l2="flushed between timed steps (256 MB write); within a step the "
                                 "weights stay L2-resident across the iterations of the decode loop", parallelism=f"replicas x{world}"),
                     clocks=clocks,

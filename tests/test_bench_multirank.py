@@ -1,0 +1,51 @@
+"""Host-side logic of the multi-process benchmark, run as two gloo ranks on the CPU: every rank decodes its own
+sentences (replicas, no collective on the data path), the job's time is the slowest rank's and its token count
+the sum; the reference arm runs on rank 0 only."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    src, lens = bench.sentence_inputs(rank)
+    t, n = bench.reduce_max_sum(dist, torch.device("cpu"), 10.0 + 5.0 * rank, 100 + rank)
+    out[rank] = (float(t), int(n), int(src.sum()), src.shape, int(lens.sum()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_sentences_and_aggregate():
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_worker, args=(2, 29533, out), nprocs=2, join=True)
+    assert out[0][:2] == (15.0, 201) and out[1][:2] == (15.0, 201)      # max over ranks, sum over ranks
+    assert out[0][3] == out[1][3] == (64, 40)
+    assert out[0][2] != out[1][2]                                       # different sentences per rank
+    sys.path.insert(0, ROOT)
+    import bench
+    a, _ = bench.sentence_inputs(0)
+    assert int(a.sum()) == out[0][2]                                    # and seeded
+
+
+def test_single_process_aggregation_is_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.reduce_max_sum(None, None, 3.5, 7) == (3.5, 7)
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
