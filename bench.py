@@ -199,7 +199,7 @@ def run_ours(args, rank, world, local_rank):
         tot = dict(accepted=0, iterations=0, kernel_launches=0, device_ms=0.0, encode_ms=0.0)
         for s in range(N_SENT):
             st = dec.generate_device(t_src[s: s + 1], t_len[s: s + 1], t_out[s: s + 1], t_olen[s: s + 1], mode="IAD", k=KMAX,
-                                     max_len_t=t_max[s: s + 1], override_t=t_str[s: s + 1])
+                                     max_len_t=t_max[s: s + 1], override_t=t_str[s: s + 1], sync_every=args.sync_every)
             for k_ in tot:
                 tot[k_] += st[k_]
         return tot
@@ -208,7 +208,8 @@ def run_ours(args, rank, world, local_rank):
         acc = 0
         for s in range(N_SENT):
             _, st = dec.generate(p_src.numpy()[s: s + 1], p_len.numpy()[s: s + 1], mode="IAD", k=KMAX, max_len=p_max.numpy()[s: s + 1],
-                                 draft_override=p_str.numpy()[s: s + 1], out=p_out.numpy()[s: s + 1], out_len=p_olen.numpy()[s: s + 1])
+                                 draft_override=p_str.numpy()[s: s + 1], out=p_out.numpy()[s: s + 1], out_len=p_olen.numpy()[s: s + 1],
+                                 sync_every=args.sync_every)
             acc += st["accepted"]
         return acc
 
@@ -330,6 +331,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sync-every", type=int, default=0, help="iterations between host checks of the finished flag (0 = library default)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work of the checker baseline sample")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

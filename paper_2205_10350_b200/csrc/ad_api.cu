@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <map>
 #include <string>
 #include <vector>
@@ -186,7 +187,7 @@ void pass_shapes(const ad_model_cfg& c, PassCfg* pass, int* M_all) {
   for (int k = 0; k < PK_COUNT; ++k) {
     pass[k].M_cap = B * pass[k].seg_max;
     pass[k].ntile = clampi(pow2ceil(pass[k].M_cap), 16, 256);
-    pass[k].max_split = pass[k].M_cap <= 256 ? 16 : 1;
+    pass[k].max_split = pass[k].M_cap <= 256 ? 16 : 4;
     if (pass[k].M_cap > all) all = pass[k].M_cap;
   }
   if (!c.has_drafter) { /* the drafter pass is never run; keep its shapes for sizing simplicity */ }
@@ -254,7 +255,7 @@ int check_cfg(const ad_model_cfg* c, std::string* why) {
   if (c->d_model > 1024) return bad("d_model must be at most 1024");
   if (c->d_ffn <= 0 || c->vocab <= 4 || c->n_enc < 1 || c->n_dec < 1) return bad("bad model sizes");
   if (c->dtype != AD_DTYPE_FP32 && c->dtype != AD_DTYPE_BF16) return bad("dtype must be AD_DTYPE_FP32 or AD_DTYPE_BF16");
-  if (c->dtype == AD_DTYPE_BF16 && (c->d_model % 64 || c->d_ffn % 64)) return bad("BF16 needs d_model and d_ffn to be multiples of 64");
+  if (c->dtype == AD_DTYPE_BF16 && (c->d_model % 128 || c->d_ffn % 64)) return bad("BF16 needs d_model to be a multiple of 128 and d_ffn a multiple of 64");
   if (c->max_batch < 1 || c->max_batch > 256) return bad("max_batch must be 1..256");
   if (c->max_src < 1 || c->max_tgt < 1) return bad("max_src and max_tgt must be positive");
   if (c->kmax < 1 || c->kmax > 256 || c->kmax > c->max_tgt) return bad("kmax must be 1..min(256, max_tgt)");
@@ -351,7 +352,9 @@ cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap&
   const int ksplit = (EPI == EPI_F32 && p.ksplit > 1) ? p.ksplit : 1;
   dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile, ksplit);
   const int stages = tc_stages(p.ntile, (p.K / tc::BLOCK_K) / ksplit, grid.x * grid.y * grid.z);
-  const size_t smem = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2) + 1024;
+  // the ring doubles as the epilogue's transposition buffer (ntile rows of 132 floats)
+  const size_t ring = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2);
+  const size_t smem = std::max(ring, (size_t)p.ntile * 132 * sizeof(float)) + 1024;
   return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(128), smem, st, mw, mx, p, stages);
 }
 

@@ -193,8 +193,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int slot_s[256];
-  __shared__ float red_val[EPI == EPI_ARGMAX ? 4 : 1][256];
-  __shared__ int red_idx[EPI == EPI_ARGMAX ? 4 : 1][256];
 
   trace_mark(TR_GEMM + EPI, 0);
   const int ntile = p.ntile;
@@ -318,10 +316,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     trace_mark(TR_GEMM + EPI, 4);
     if (EPI == EPI_SCATTER) __syncthreads();   // slot_s visible (every thread reaches this point)
+    // The accumulator holds one output feature per thread (TMEM lane) and one token per column.  It is first
+    // transposed through shared memory (the TMA ring is free once the accumulator barrier has fired) into rows
+    // of 128 features per token, so that global stores are 16 bytes per thread and whole 128-feature rows
+    // per warp, and so that the arg-max scan of a token needs no shuffles.
+    float* stage = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+    constexpr int LD = (EPI == EPI_ARGMAX) ? 129 : 132;   // 129: conflict-free column scans; 132: 16-byte aligned rows
+    const int ntok = min(ntile, M - t0);                   // valid tokens of this tile (<= 0 only if M == 0)
     if (ready) {
-      float* out_f32 = (EPI == EPI_F32) ? p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N : nullptr;
       for (int c = 0; c < ntile; c += 32) {
-        if (t0 + c >= M) break;
+        if (c >= ntok) break;
         float acc[32];
         const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c);
         if (ntile - c >= 32) {
@@ -331,40 +335,97 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
           for (int j = 16; j < 32; ++j) acc[j] = 0.f;
         }
-        if (EPI == EPI_ARGMAX) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (c + j < ntile && t0 + c + j < M) {      // uniform over the warp
-              // features grow with the lane, so the lowest winning lane is the lowest winning id
-              float best;
-              int wl;
-              warp_argmax_lane((n < p.N) ? acc[j] : -INFINITY, best, wl);
-              if (lane == 0) { red_val[warp][c + j] = best; red_idx[warp][c + j] = n0 + warp * 32 + wl; }
-            }
+        for (int j = 0; j < 32; ++j) {
+          if (c + j < ntok) {
+            float v = acc[j] + bias_n;
+            if (EPI == EPI_ACT && p.relu) v = fmaxf(v, 0.f);
+            if (EPI == EPI_ARGMAX && n >= p.N) v = -INFINITY;
+            stage[(c + j) * LD + threadIdx.x] = v;
           }
-        } else {
-          epilogue_chunk<EPI, bf16>(p, n, t0 + c, M, acc, bias_n, out_f32, slot_s, c);
-          if (ntile - c >= 32) epilogue_chunk<EPI, bf16>(p, n, t0 + c + 16, M, acc + 16, bias_n, out_f32, slot_s, c + 16);
         }
       }
     }
     trace_mark(TR_GEMM + EPI, 5);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (EPI == EPI_ARGMAX && ready) {
-      for (int j = threadIdx.x; j < ntile; j += blockDim.x) {
-        const int m = t0 + j;
-        if (m < M) {
-          float v = red_val[0][j];
-          int i = red_idx[0][j];
-#pragma unroll
-          for (int w = 1; w < 4; ++w) {
-            const float ov = red_val[w][j];
-            const int oi = red_idx[w][j];
-            if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+    if (ready && ntok > 0) {
+      if (EPI == EPI_F32) {
+        float* out = p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N;
+        const int col = n0 + lane * 4;
+        const bool vec = (p.N & 3) == 0;
+        for (int r = warp; r < ntok; r += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(stage + r * LD + lane * 4);
+          float* dst = out + (size_t)(t0 + r) * p.N + col;
+          if (vec && col + 3 < p.N) {
+            *reinterpret_cast<float4*>(dst) = v;
+          } else {
+            if (col < p.N) dst[0] = v.x;
+            if (col + 1 < p.N) dst[1] = v.y;
+            if (col + 2 < p.N) dst[2] = v.z;
+            if (col + 3 < p.N) dst[3] = v.w;
           }
-          p.part_val[(size_t)blockIdx.x * p.M_cap + m] = v;
-          p.part_idx[(size_t)blockIdx.x * p.M_cap + m] = i;
+        }
+      } else if (EPI == EPI_ACT || EPI == EPI_SCATTER) {
+        // two token rows per warp pass: 16 lanes x 8 features = 128 features = 256 bytes of bf16
+        const int half = lane >> 4, f0 = (lane & 15) * 8;
+        int width = p.N, seg = 0, col0 = n0;
+        bf16* base = reinterpret_cast<bf16*>(p.out_act);
+        if (EPI == EPI_SCATTER) {           // a 128-feature tile lies inside one segment (seg_width % 128 == 0)
+          width = p.seg_width;
+          seg = n0 / width;
+          col0 = n0 - seg * width;
+          base = reinterpret_cast<bf16*>(p.dst[seg]);
+        }
+        const bool vec = (width & 7) == 0;
+        for (int r = warp * 2 + half; r < ntok; r += 8) {
+          const float* srow = stage + r * LD + f0;
+          const float4 a = *reinterpret_cast<const float4*>(srow);
+          const float4 b = *reinterpret_cast<const float4*>(srow + 4);
+          const int grow = (EPI == EPI_SCATTER && seg >= p.n_direct) ? slot_s[r] : t0 + r;
+          bf16* dst = base + (size_t)grow * width + col0 + f0;
+          const int lim = p.N - (n0 + f0);                 // features of this lane that exist
+          if (vec && lim >= 8) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+            uint4 u;
+            u.x = *reinterpret_cast<unsigned int*>(&h0); u.y = *reinterpret_cast<unsigned int*>(&h1);
+            u.z = *reinterpret_cast<unsigned int*>(&h2); u.w = *reinterpret_cast<unsigned int*>(&h3);
+            *reinterpret_cast<uint4*>(dst) = u;
+          } else {
+            const float vals[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+              if (t < lim) dst[t] = __float2bfloat16_rn(vals[t]);
+          }
+        }
+      } else {
+        // EPI_ARGMAX: `parts` threads share a token, each scanning 128 / parts consecutive features in
+        // ascending order (strict > keeps the lowest id); the parts are then combined in ascending order too.
+        const int parts = ntile >= 128 ? 1 : 128 / ntile;
+        const int per = 128 / parts;
+        for (int base_tok = 0; base_tok < ntok; base_tok += 128 / parts) {
+          const int tok = base_tok + (int)threadIdx.x / parts, part = (int)threadIdx.x % parts;
+          float v = -INFINITY;
+          int idx = 0;
+          if (tok < ntok) {
+            const float* srow = stage + tok * LD + part * per;
+            for (int f = 0; f < per; ++f) {
+              const float x = srow[f];
+              if (x > v) { v = x; idx = f; }
+            }
+            idx += n0 + part * per;
+          }
+          // combine the parts of a token: they sit in consecutive lanes (parts is a power of two <= 8)
+          for (int o = 1; o < parts; o <<= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+          }
+          if (tok < ntok && part == 0) {
+            p.part_val[(size_t)blockIdx.x * p.M_cap + t0 + tok] = v;
+            p.part_idx[(size_t)blockIdx.x * p.M_cap + t0 + tok] = idx;
+          }
         }
       }
     }
