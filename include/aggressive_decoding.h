@@ -102,7 +102,7 @@ typedef struct ad_gen_opts {
   int32_t run_drafter;   /* GAD only: 1 = run the drafter forward every iteration (its block is then replaced by
                             draft_override when that is given); 0 = skip it (needs draft_override) */
   int32_t sync_every;    /* iterations between host checks of the device-side "all rows finished" word;
-                            0 = library default */
+                            0 = library default (1) */
   int32_t use_graph;     /* 1 = replay one captured CUDA graph per iteration, 0 = launch kernels directly.
                             Ignored (direct launches) when the handle was created on the default stream,
                             which cannot be captured. */
@@ -201,6 +201,12 @@ int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_
 
 /* Debug: FP32 copy of the verifier's encoder memory of row b, [src_len_b, d_model] (device pointer). */
 int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size_t capacity_elems);
+
+/* Debug: exercises the bounded-wait mechanism that every mbarrier wait of the GEMM kernels uses.  Launches one
+ * tiny kernel that polls, at most poll_limit (1..65536) times, a barrier phase that nothing completes; the wait
+ * runs out, AD_ERR_TIMEOUT is latched in *status (device int, must be 0 before) and the kernel returns
+ * normally, leaving the context usable.  polls_done (device int, may be NULL) receives the number of polls. */
+int ad_debug_wait_probe(int32_t* status, int32_t poll_limit, int32_t* polls_done, void* stream);
 
 /* ---- single-kernel entry points (operator-level tests and microbenchmarks) --------------------------
  * All pointers are device pointers; `stream` is a cudaStream_t.  Asynchronous. */

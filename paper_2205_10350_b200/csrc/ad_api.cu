@@ -878,7 +878,7 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
     }
   }
 
-  const int sync_every = opts->sync_every > 0 ? opts->sync_every : 4;
+  const int sync_every = opts->sync_every > 0 ? opts->sync_every : 1;
   int iters = 0;
   volatile int* flag = h->host_flag;
   flag[0] = 0;
@@ -950,6 +950,30 @@ extern "C" int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size
   else to_f32_kernel<float><<<64, 256, 0, h->stream>>>((const float*)h->encmem + start, mem, n);
   AD_CUDA(h, cudaGetLastError());
   return AD_OK;
+}
+
+// ---- bounded-wait self-test ---------------------------------------------------------------------------
+
+namespace {
+// One thread waits, with the given poll limit, on an mbarrier phase that nothing ever completes.
+__global__ void wait_probe_kernel(int* status, unsigned int limit, int* polls_done) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    unsigned int i = 0;
+    bool done = false;
+    for (; i < limit && !done; ++i) done = tc::mbar_try_wait(tc::smem_u32(&bar), 0);
+    if (!done) latch_error(status, AD_ERR_TIMEOUT);
+    if (polls_done) *polls_done = (int)i;
+  }
+}
+}  // namespace
+
+extern "C" int ad_debug_wait_probe(int32_t* status, int32_t poll_limit, int32_t* polls_done, void* stream) {
+  if (!status || poll_limit < 1 || poll_limit > (1 << 16)) return AD_ERR_ARG;
+  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, (unsigned int)poll_limit, polls_done);
+  return cudaGetLastError() == cudaSuccess ? AD_OK : AD_ERR_CUDA;
 }
 
 // ---- single-kernel entry points -----------------------------------------------------------------
