@@ -390,6 +390,18 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   return AD_OK;
 }
 
+template <typename T, int D, int Q>
+cudaError_t launch_attention(dim3 grid, dim3 block, cudaStream_t st, const AttnParams& p) {
+  constexpr size_t smem = att_smem_bytes<D, Q>();
+  static bool attr_set = false;
+  if (!attr_set && smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  attr_set = true;
+  return launch_k(attention_kernel<T, D, Q>, grid, block, smem, st, p);
+}
+
 int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, const void* v, void* out,
               const int* key_base, const int* nkeys_tok, const int* nkeys_row) {
   const ad_model_cfg& c = h->cfg;
@@ -398,20 +410,25 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   p.seg_off = pc.plan.seg_off; p.seg_len = pc.plan.seg_len;
   p.key_base = key_base; p.nkeys_tok = nkeys_tok; p.nkeys_row = nkeys_row;
   p.d = c.d_model;
-  p.qchunks = (pc.seg_max + ATT_QC - 1) / ATT_QC;
+  // one query per warp while the grid stays within a couple of waves, eight when there are many queries
   const int dh = c.d_model / c.n_heads;
+  const bool many = (long long)h->dims.B * c.n_heads * ((pc.seg_max + 7) / 8) > 3LL * num_sms();
+  const int qpw = many ? 8 : 1;
+  p.qchunks = (pc.seg_max + 8 * qpw - 1) / (8 * qpw);
   p.scale = 1.0f / sqrtf((float)dh);
   dim3 grid(h->dims.B * p.qchunks, c.n_heads);
   const dim3 block(256);
   h->launches++;
   cudaError_t e;
+#define AD_ATT(T, D, Q) launch_attention<T, D, Q>(grid, block, h->stream, p)
   if (h->bf16) {
-    if (dh == 64) e = launch_k(attention_kernel<bf16, 64>, grid, block, 0, h->stream, p);
-    else e = launch_k(attention_kernel<bf16, 32>, grid, block, 0, h->stream, p);
+    if (dh == 64) e = many ? AD_ATT(bf16, 64, 8) : AD_ATT(bf16, 64, 1);
+    else e = many ? AD_ATT(bf16, 32, 8) : AD_ATT(bf16, 32, 1);
   } else {
-    if (dh == 64) e = launch_k(attention_kernel<float, 64>, grid, block, 0, h->stream, p);
-    else e = launch_k(attention_kernel<float, 32>, grid, block, 0, h->stream, p);
+    if (dh == 64) e = many ? AD_ATT(float, 64, 8) : AD_ATT(float, 64, 1);
+    else e = many ? AD_ATT(float, 32, 8) : AD_ATT(float, 32, 1);
   }
+#undef AD_ATT
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
   return AD_OK;
 }

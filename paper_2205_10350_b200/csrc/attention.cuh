@@ -24,7 +24,7 @@ struct AttnParams {
   const int* nkeys_tok;  // [M_cap] keys visible to each packed token, or null
   const int* nkeys_row;  // [B] upper bound of the keys any token of row b sees (the count itself when nkeys_tok is null)
   int d;
-  int qchunks;           // query chunks per row = ceil(longest possible segment / 16)
+  int qchunks;           // query chunks per row = ceil(longest possible segment / queries per CTA)
   float scale;           // 1 / sqrt(head dim)
 };
 
@@ -46,20 +46,30 @@ __device__ __forceinline__ void load8(const float* p, float* out) {
   out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
 }
 
-constexpr int ATT_QC = 8;    // queries per CTA: one per warp
-constexpr int ATT_KT = 64;   // keys per shared-memory tile
+constexpr int ATT_WARPS = 8;   // warps per CTA
+constexpr int ATT_KT = 64;     // keys per shared-memory tile
 
-// grid = (B * qchunks, H); block = 256 threads (8 warps, one query each).
+template <int DH, int QPW>
+constexpr size_t att_smem_bytes() {
+  return sizeof(float) * (size_t)(ATT_KT * (DH + 1) + ATT_KT * DH + ATT_WARPS * QPW * DH + ATT_WARPS * QPW * ATT_KT);
+}
+
+// grid = (B * qchunks, H); block = 256 threads (8 warps, QPW queries each; a CTA covers 8 * QPW queries of one
+// row and one head and stages every K/V tile once for all of them).  QPW = 1 keeps the critical path short when
+// there are few queries; QPW = 8 amortises the K/V staging when there are thousands.
 // Global-memory round trips on the critical path: (1) the row's segment / key-range descriptors,
 // (2) the queries, their key counts and the first K/V tile together, then compute and store.
-template <typename ActT, int DH>
+template <typename ActT, int DH, int QPW>
 __global__ void __launch_bounds__(256)
 attention_kernel(const AttnParams p) {
   constexpr int R = DH / 32;                 // output dims per lane
-  __shared__ float ks[ATT_KT][DH + 1];
-  __shared__ float vs[ATT_KT][DH];
-  __shared__ float qs[ATT_QC][DH];
-  __shared__ float ps[ATT_QC][ATT_KT];
+  constexpr int QC = ATT_WARPS * QPW;        // queries per CTA
+  // dynamic shared memory (att_smem_bytes<DH, QPW>()): K tile (padded rows), V tile, queries, probabilities
+  extern __shared__ __align__(16) float att_smem[];
+  float (*ks)[DH + 1] = reinterpret_cast<float (*)[DH + 1]>(att_smem);
+  float (*vs)[DH] = reinterpret_cast<float (*)[DH]>(att_smem + ATT_KT * (DH + 1));
+  float (*qs)[DH] = reinterpret_cast<float (*)[DH]>(att_smem + ATT_KT * (DH + 1) + ATT_KT * DH);
+  float (*ps)[ATT_KT] = reinterpret_cast<float (*)[ATT_KT]>(att_smem + ATT_KT * (DH + 1) + ATT_KT * DH + QC * DH);
 
   trace_mark(TR_ATTN, 0);
   pdl_launch();
@@ -72,29 +82,37 @@ attention_kernel(const AttnParams p) {
   const int seg_off = p.seg_off[b];
   const int kbase = p.key_base[b];
   const int row_nk = p.nkeys_row[b];         // no token of this row sees more keys than this
-  const int i0 = chunk * ATT_QC;
+  const int i0 = chunk * QC;
   if (i0 >= seg_len) return;
-  const int nq = min(ATT_QC, seg_len - i0);
+  const int nq = min(QC, seg_len - i0);
   const int m0 = seg_off + i0;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const ActT* q = reinterpret_cast<const ActT*>(p.q);
   const ActT* kk = reinterpret_cast<const ActT*>(p.k);
   const ActT* vv = reinterpret_cast<const ActT*>(p.v);
   const int d = p.d;
-  const bool has_q = warp < nq;
 
-  // this warp's query and its visible-key count
-  int nk = 0;
-  if (has_q) {
-    nk = p.nkeys_tok ? min(p.nkeys_tok[m0 + warp], row_nk) : row_nk;
+  // this warp's queries (warp, warp + 8, ...) and their visible-key counts
+  int nk[QPW];
 #pragma unroll
-    for (int rr = 0; rr < R; ++rr)
-      qs[warp][lane + 32 * rr] = to_f32(q[(size_t)(m0 + warp) * d + h * DH + lane + 32 * rr]) * p.scale;
+  for (int t = 0; t < QPW; ++t) {
+    const int r = warp + ATT_WARPS * t;
+    nk[t] = 0;
+    if (r < nq) {
+      nk[t] = p.nkeys_tok ? min(p.nkeys_tok[m0 + r], row_nk) : row_nk;
+#pragma unroll
+      for (int rr = 0; rr < R; ++rr)
+        qs[r][lane + 32 * rr] = to_f32(q[(size_t)(m0 + r) * d + h * DH + lane + 32 * rr]) * p.scale;
+    }
   }
 
-  float mx = -INFINITY, den = 0.f, acc[R];
+  float mx[QPW], den[QPW], acc[QPW][R];
 #pragma unroll
-  for (int r = 0; r < R; ++r) acc[r] = 0.f;
+  for (int t = 0; t < QPW; ++t) {
+    mx[t] = -INFINITY; den[t] = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[t][r] = 0.f;
+  }
 
   for (int j0 = 0; j0 < row_nk; j0 += ATT_KT) {
     __syncthreads();   // previous tile fully consumed
@@ -113,47 +131,74 @@ attention_kernel(const AttnParams p) {
       for (int t = 0; t < 8; ++t) { ks[j][c + t] = kf[t]; vs[j][c + t] = vf[t]; }
     }
     __syncthreads();
-    if (nk <= j0) continue;   // warp-uniform: no visible key in this tile (the barriers above are still reached)
-    float s0 = 0.f, s1 = 0.f;
-#pragma unroll 8
+    // scores of this warp's QPW queries against keys lane and lane + 32: every K element read from shared
+    // memory is used for all QPW queries
+    float s0[QPW], s1[QPW];
+#pragma unroll
+    for (int t = 0; t < QPW; ++t) { s0[t] = 0.f; s1[t] = 0.f; }
+#pragma unroll 4
     for (int c = 0; c < DH; ++c) {
-      const float qv = qs[warp][c];
-      s0 = fmaf(qv, ks[lane][c], s0);
-      s1 = fmaf(qv, ks[lane + 32][c], s1);
+      const float k0 = ks[lane][c], k1 = ks[lane + 32][c];
+#pragma unroll
+      for (int t = 0; t < QPW; ++t) {
+        const float qv = qs[warp + ATT_WARPS * t][c];
+        s0[t] = fmaf(qv, k0, s0[t]);
+        s1[t] = fmaf(qv, k1, s1[t]);
+      }
     }
-    if (j0 + lane >= nk) s0 = -INFINITY;
-    if (j0 + lane + 32 >= nk) s1 = -INFINITY;
-    float tmax = fmaxf(s0, s1);
+    float corr[QPW];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
-    const float m_new = fmaxf(mx, tmax);           // finite: key j0 is visible
-    const float corr = expf(mx - m_new);           // exp(-inf) = 0 on the first tile
-    const float p0 = expf(s0 - m_new), p1 = expf(s1 - m_new);
-    float psum = p0 + p1;
+    for (int t = 0; t < QPW; ++t) {
+      float p0 = 0.f, p1 = 0.f;
+      corr[t] = 1.f;
+      if (nk[t] > j0) {              // warp-uniform; otherwise no key of this tile is visible to the query
+        const float a0 = (j0 + lane < nk[t]) ? s0[t] : -INFINITY;
+        const float a1 = (j0 + lane + 32 < nk[t]) ? s1[t] : -INFINITY;
+        float tmax = fmaxf(a0, a1);
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, off);
-    den = den * corr + psum;
-    mx = m_new;
-    ps[warp][lane] = p0;
-    ps[warp][lane + 32] = p1;
+        for (int off = 16; off > 0; off >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
+        const float m_new = fmaxf(mx[t], tmax);        // finite: key j0 is visible
+        corr[t] = expf(mx[t] - m_new);                 // exp(-inf) = 0 on the first tile
+        p0 = expf(a0 - m_new);
+        p1 = expf(a1 - m_new);
+        float psum = p0 + p1;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, off);
+        den[t] = den[t] * corr[t] + psum;
+        mx[t] = m_new;
+      }
+      ps[warp * QPW + t][lane] = p0;
+      ps[warp * QPW + t][lane + 32] = p1;
+    }
     __syncwarp();
 #pragma unroll
     for (int rr = 0; rr < R; ++rr) {
-      float a = acc[rr] * corr;
       const int c = lane + 32 * rr;
-#pragma unroll 8
-      for (int j = 0; j < ATT_KT; ++j) a = fmaf(ps[warp][j], vs[j][c], a);
-      acc[rr] = a;
+      float a[QPW];
+#pragma unroll
+      for (int t = 0; t < QPW; ++t) a[t] = acc[t][rr] * corr[t];
+#pragma unroll 4
+      for (int j = 0; j < ATT_KT; ++j) {
+        const float v = vs[j][c];
+#pragma unroll
+        for (int t = 0; t < QPW; ++t) a[t] = fmaf(ps[warp * QPW + t][j], v, a[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < QPW; ++t) acc[t][rr] = a[t];
     }
     __syncwarp();
   }
 
-  if (has_q && nk > 0) {
-    ActT* out = reinterpret_cast<ActT*>(p.out);
-    const float inv = 1.f / den;
+  ActT* out = reinterpret_cast<ActT*>(p.out);
 #pragma unroll
-    for (int rr = 0; rr < R; ++rr)
-      out[(size_t)(m0 + warp) * d + h * DH + lane + 32 * rr] = from_f32<ActT>(acc[rr] * inv);
+  for (int t = 0; t < QPW; ++t) {
+    const int r = warp + ATT_WARPS * t;
+    if (r < nq && nk[t] > 0) {
+      const float inv = 1.f / den[t];
+#pragma unroll
+      for (int rr = 0; rr < R; ++rr)
+        out[(size_t)(m0 + r) * d + h * DH + lane + 32 * rr] = from_f32<ActT>(acc[t][rr] * inv);
+    }
   }
   trace_mark(TR_ATTN, 2);
 }
