@@ -336,7 +336,7 @@ int num_sms() {
 // whole grid is resident at once.
 int tc_stages(int ntile, int kb, int n_ctas) {
   const int stage = tc::A_STAGE_BYTES + ntile * tc::BLOCK_K * 2;
-  const int budget = (ntile <= 64 && n_ctas > num_sms()) ? 100 * 1024 : 200 * 1024;
+  const int budget = ((ntile <= 64 && n_ctas > num_sms()) || n_ctas > 2 * num_sms()) ? 100 * 1024 : 200 * 1024;
   int s = clampi(budget / stage, 1, tc::MAX_STAGES);
   return s < kb ? s : (kb > 0 ? kb : 1);
 }
@@ -352,9 +352,9 @@ cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap&
   const int ksplit = (EPI == EPI_F32 && p.ksplit > 1) ? p.ksplit : 1;
   dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile, ksplit);
   const int stages = tc_stages(p.ntile, (p.K / tc::BLOCK_K) / ksplit, grid.x * grid.y * grid.z);
-  // the ring doubles as the epilogue's transposition buffer (ntile rows of 132 floats)
+  // the ring doubles as the epilogue's transposition buffer (up to 128 rows of 132 floats)
   const size_t ring = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2);
-  const size_t smem = std::max(ring, (size_t)p.ntile * 132 * sizeof(float)) + 1024;
+  const size_t smem = std::max(ring, (size_t)std::min(p.ntile, 128) * 132 * sizeof(float)) + 1024;
   return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(128), smem, st, mw, mx, p, stages);
 }
 

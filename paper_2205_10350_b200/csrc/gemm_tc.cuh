@@ -270,9 +270,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     if (lane == 0 && warp != 1) {
       // ---- TMA producers: everything that was not issued above ----
+      // No more producers than stages: a producer's consecutive K blocks are then at most one ring round apart,
+      // so its parity wait on an "empty" barrier can never alias a phase two rounds back.
       const int pw = warp == 0 ? 0 : warp - 1;          // 0, 1, 2
+      const int nprod = stages < 3 ? stages : 3;
       const int begin = early ? first_round : 0;
-      for (int i = begin + pw; i < num_kb; i += 3) {
+      for (int i = begin + pw; pw < nprod && i < num_kb; i += nprod) {
         const int s = i % stages;
         const uint32_t round = i / stages;
         if (round > 0 && !mbar_wait(smem_u32(&bar_empty[s]), (round - 1) & 1, p.status)) { abort_flag = 1; break; }
@@ -322,15 +325,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // per warp, and so that the arg-max scan of a token needs no shuffles.
     float* stage = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
     constexpr int LD = (EPI == EPI_ARGMAX) ? 129 : 132;   // 129: conflict-free column scans; 132: 16-byte aligned rows
-    const int ntok = min(ntile, M - t0);                   // valid tokens of this tile (<= 0 only if M == 0)
-    if (ready) {
-      for (int c = 0; c < ntile; c += 32) {
+    const int ntok_all = min(ntile, M - t0);               // valid tokens of this tile (<= 0 only if M == 0)
+    const int sub = ntile < 128 ? ntile : 128;             // tokens transposed per pass (bounds the buffer to 68 KB)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    for (int tb = 0; tb < ntile && tb < ntok_all && ready; tb += sub) {
+      const int ntok = min(sub, ntok_all - tb);            // valid tokens of this pass
+      const int tg = t0 + tb;                              // packed index of the pass's first token
+      if (tb > 0) __syncthreads();                         // previous pass has been read out
+      for (int c = 0; c < sub; c += 32) {
         if (c >= ntok) break;
         float acc[32];
-        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(c);
-        if (ntile - c >= 32) {
+        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(tb + c);
+        if (sub - c >= 32) {
           tmem_ld32(taddr, acc);
-        } else {          // ntile == 16
+        } else {          // 16-token tile
           tmem_ld16(taddr, acc);
 #pragma unroll
           for (int j = 16; j < 32; ++j) acc[j] = 0.f;
@@ -345,18 +353,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           }
         }
       }
-    }
-    trace_mark(TR_GEMM + EPI, 5);
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (ready && ntok > 0) {
+      if (tb == 0) trace_mark(TR_GEMM + EPI, 5);
+      __syncthreads();
       if (EPI == EPI_F32) {
         float* out = p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N;
         const int col = n0 + lane * 4;
         const bool vec = (p.N & 3) == 0;
         for (int r = warp; r < ntok; r += 4) {
           const float4 v = *reinterpret_cast<const float4*>(stage + r * LD + lane * 4);
-          float* dst = out + (size_t)(t0 + r) * p.N + col;
+          float* dst = out + (size_t)(tg + r) * p.N + col;
           if (vec && col + 3 < p.N) {
             *reinterpret_cast<float4*>(dst) = v;
           } else {
@@ -382,7 +387,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           const float* srow = stage + r * LD + f0;
           const float4 a = *reinterpret_cast<const float4*>(srow);
           const float4 b = *reinterpret_cast<const float4*>(srow + 4);
-          const int grow = (EPI == EPI_SCATTER && seg >= p.n_direct) ? slot_s[r] : t0 + r;
+          const int grow = (EPI == EPI_SCATTER && seg >= p.n_direct) ? slot_s[tb + r] : tg + r;
           bf16* dst = base + (size_t)grow * width + col0 + f0;
           const int lim = p.N - (n0 + f0);                 // features of this lane that exist
           if (vec && lim >= 8) {
@@ -402,33 +407,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       } else {
         // EPI_ARGMAX: `parts` threads share a token, each scanning 128 / parts consecutive features in
         // ascending order (strict > keeps the lowest id); the parts are then combined in ascending order too.
-        const int parts = ntile >= 128 ? 1 : 128 / ntile;
+        const int parts = 128 / sub;
         const int per = 128 / parts;
-        for (int base_tok = 0; base_tok < ntok; base_tok += 128 / parts) {
-          const int tok = base_tok + (int)threadIdx.x / parts, part = (int)threadIdx.x % parts;
-          float v = -INFINITY;
-          int idx = 0;
-          if (tok < ntok) {
-            const float* srow = stage + tok * LD + part * per;
-            for (int f = 0; f < per; ++f) {
-              const float x = srow[f];
-              if (x > v) { v = x; idx = f; }
-            }
-            idx += n0 + part * per;
+        const int tok = (int)threadIdx.x / parts, part = (int)threadIdx.x % parts;
+        float v = -INFINITY;
+        int idx = 0;
+        if (tok < ntok) {
+          const float* srow = stage + tok * LD + part * per;
+          for (int f = 0; f < per; ++f) {
+            const float x = srow[f];
+            if (x > v) { v = x; idx = f; }
           }
-          // combine the parts of a token: they sit in consecutive lanes (parts is a power of two <= 8)
-          for (int o = 1; o < parts; o <<= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-            if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-          }
-          if (tok < ntok && part == 0) {
-            p.part_val[(size_t)blockIdx.x * p.M_cap + t0 + tok] = v;
-            p.part_idx[(size_t)blockIdx.x * p.M_cap + t0 + tok] = idx;
-          }
+          idx += n0 + part * per;
+        }
+        // combine the parts of a token: they sit in consecutive lanes (parts is a power of two <= 8)
+        for (int o = 1; o < parts; o <<= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+          if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+        }
+        if (tok < ntok && part == 0) {
+          p.part_val[(size_t)blockIdx.x * p.M_cap + tg + tok] = v;
+          p.part_idx[(size_t)blockIdx.x * p.M_cap + tg + tok] = idx;
         }
       }
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
   }
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
