@@ -30,7 +30,8 @@ struct Mat {
 struct ActBuf {
   void* ptr = nullptr;
   int cols = 0;
-  CUtensorMap map[PK_COUNT];
+  CUtensorMap map[PK_COUNT];        // box rows = the pass's token tile
+  CUtensorMap map_half[PK_COUNT];   // box rows = half of it (used when the full tile would leave most SMs idle)
 };
 struct EncLayer {
   Mat wqkv, wo, w1, w2;
@@ -56,8 +57,14 @@ struct PassCfg {
   PassPlan plan;
   // Split-K factor of a projection that feeds the LayerNorm kernel: enough CTAs to cover the SMs when the
   // token dimension alone gives only a handful of tiles (power of two, divides the K blocks, <= max_split).
-  int ksplit_for(int N, int K) const {
-    const int tiles = ((N + 127) / 128) * ((M_cap + ntile - 1) / ntile);
+  // Token tile for a projection with N output features: the pass's tile, or half of a 256-token tile when the
+  // full tile would give fewer CTAs than two per SM (the K loop costs the same per CTA either way).
+  int tile_for(int N, int n_sms) const {
+    if (ntile == 256 && ((N + 127) / 128) * ((M_cap + 255) / 256) < 2 * n_sms) return 128;
+    return ntile;
+  }
+  int ksplit_for(int N, int K, int tile) const {
+    const int tiles = ((N + 127) / 128) * ((M_cap + tile - 1) / tile);
     const int kb = K / 64;
     int s = 1;
     while (s * 2 <= max_split && tiles * s * 2 <= 160 && kb % (s * 2) == 0) s *= 2;
@@ -369,13 +376,14 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   cudaError_t e;
   h->launches++;
   if (h->bf16) {
-    p.ntile = h->pass[pk].ntile;
+    p.ntile = h->pass[pk].tile_for(W.N, num_sms());
+    const CUtensorMap& mx = (p.ntile == h->pass[pk].ntile) ? X.map[pk] : X.map_half[pk];
     if (epi != EPI_F32) p.ksplit = 1;
     switch (epi) {
-      case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, X.map[pk], p, M_cap); break;
-      case EPI_ACT: e = launch_tc<EPI_ACT>(h->stream, W.map, X.map[pk], p, M_cap); break;
-      case EPI_SCATTER: e = launch_tc<EPI_SCATTER>(h->stream, W.map, X.map[pk], p, M_cap); break;
-      default: e = launch_tc<EPI_ARGMAX>(h->stream, W.map, X.map[pk], p, M_cap); break;
+      case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, mx, p, M_cap); break;
+      case EPI_ACT: e = launch_tc<EPI_ACT>(h->stream, W.map, mx, p, M_cap); break;
+      case EPI_SCATTER: e = launch_tc<EPI_SCATTER>(h->stream, W.map, mx, p, M_cap); break;
+      default: e = launch_tc<EPI_ARGMAX>(h->stream, W.map, mx, p, M_cap); break;
     }
   } else {
     p.ntile = simt::TOK;
@@ -454,7 +462,7 @@ int gemm_to_ln(ad_handle* h, const Mat& W, const ActBuf& X, int pk, int* nsplit)
   PassCfg& pc = h->pass[pk];
   GemmParams o = {};
   o.out_f32 = h->pre;
-  o.ksplit = h->bf16 ? pc.ksplit_for(W.N, W.K) : 1;
+  o.ksplit = h->bf16 ? pc.ksplit_for(W.N, W.K, pc.tile_for(W.N, num_sms())) : 1;
   *nsplit = o.ksplit;
   return gemm(h, EPI_F32, W, X, pk, pc.plan.M, pc.M_cap, o);
 }
@@ -683,7 +691,10 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
     bool ok = true;
     ActBuf* bufs[4] = {&h->yb, &h->abuf, &h->hbuf, &h->xg};
     for (ActBuf* b : bufs)
-      for (int k = 0; k < PK_COUNT; ++k) ok = ok && make_map(&b->map[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile);
+      for (int k = 0; k < PK_COUNT; ++k) {
+        ok = ok && make_map(&b->map[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile);
+        ok = ok && make_map(&b->map_half[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile / 2);
+      }
     if (!ok) return bail(AD_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   }
   // Cache, scratch and state start from zero so that no stale bit pattern is ever read as a number.
@@ -1009,8 +1020,8 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part_val, const int
   float v = -INFINITY;
   int idx = 0x7fffffff;
   for (int t = lane; t < n_tiles; t += 32) {
-    const float ov = part_val[(size_t)t * M_cap + m];
-    const int oi = part_idx[(size_t)t * M_cap + m];
+    const float ov = part_val[(size_t)m * n_tiles + t];
+    const int oi = part_idx[(size_t)m * n_tiles + t];
     if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
   }
   tc::warp_argmax(v, idx);

@@ -68,8 +68,8 @@ struct GemmParams {
   int n_direct;
   const int* slot;       // [M_cap]
   // EPI_ARGMAX
-  float* part_val;       // [n_tiles, M_cap]
-  int* part_idx;         // [n_tiles, M_cap]
+  float* part_val;       // [M_cap, n_tiles]: per token, the best value of every 128-feature tile
+  int* part_idx;         // [M_cap, n_tiles]
   int* status;           // device status word (latches AD_ERR_TIMEOUT), may be null
 };
 

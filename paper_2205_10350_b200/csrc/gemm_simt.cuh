@@ -80,8 +80,8 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
         const int oi = red_idx[wq][tid];
         if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
       }
-      p.part_val[(size_t)blockIdx.x * p.M_cap + t0 + tid] = v;
-      p.part_idx[(size_t)blockIdx.x * p.M_cap + t0 + tid] = i;
+      p.part_val[(size_t)(t0 + tid) * gridDim.x + blockIdx.x] = v;
+      p.part_idx[(size_t)(t0 + tid) * gridDim.x + blockIdx.x] = i;
     }
   } else {
     __shared__ int slot_s[TOK];

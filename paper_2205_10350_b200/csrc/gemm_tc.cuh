@@ -427,8 +427,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
         }
         if (tok < ntok && part == 0) {
-          p.part_val[(size_t)blockIdx.x * p.M_cap + tg + tok] = v;
-          p.part_idx[(size_t)blockIdx.x * p.M_cap + tg + tok] = idx;
+          p.part_val[(size_t)(tg + tok) * gridDim.x + blockIdx.x] = v;
+          p.part_idx[(size_t)(tg + tok) * gridDim.x + blockIdx.x] = idx;
         }
       }
     }

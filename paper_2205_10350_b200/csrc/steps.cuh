@@ -460,8 +460,8 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
       float v = -INFINITY;
       int idx = 0x7fffffff;
       for (int t = lane; t < n_tiles; t += 32) {
-        const float ov = part_val[(size_t)t * M_cap + m];
-        const int oi = part_idx[(size_t)t * M_cap + m];
+        const float ov = part_val[(size_t)m * n_tiles + t];
+        const int oi = part_idx[(size_t)m * n_tiles + t];
         if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
       }
 #pragma unroll
