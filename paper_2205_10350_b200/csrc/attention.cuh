@@ -177,8 +177,9 @@ attention_kernel(const AttnParams p) {
       float a[QPW];
 #pragma unroll
       for (int t = 0; t < QPW; ++t) a[t] = acc[t][rr] * corr[t];
+      const int jn = min(ATT_KT, row_nk - j0);      // keys of this tile that exist at all
 #pragma unroll 4
-      for (int j = 0; j < ATT_KT; ++j) {
+      for (int j = 0; j < jn; ++j) {
         const float v = vs[j][c];
 #pragma unroll
         for (int t = 0; t < QPW; ++t) a[t] = fmaf(ps[warp * QPW + t][j], v, a[t]);
