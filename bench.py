@@ -38,7 +38,7 @@ KMAX = 40                      # outputs are at most 40 tokens, so the block cap
 METRIC, UNIT = "verified_tokens_per_s", "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the projection kernel at this exact shape
 # (profiles/vocab_argmax_gemm_base_M40_ncu_full.txt); set to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES = 32849664
+NCU_TRAFFIC_BYTES = 32840960
 WORKLOAD_DESC = ("transformer-base (6+6, d512, h8, ffn2048, vocab 32000, bf16) GEC-shaped input-guided decoding, batch 1, "
                  "source length U[12,40], drafts = own greedy output with 10% of tokens replaced, block = remaining "
                  "length (cap 64 never binds)")
@@ -273,17 +273,18 @@ def run_ours(args, rank, world, local_rank):
         assert rc == 0
 
     def time_vocab(cold, reps=20):
-        ts = []
+        # everything is enqueued first and the stream synchronised once, so that the events bracket device time
+        # only (a host round trip per launch would add the launch latency to every sample)
+        evs = []
         with torch.cuda.stream(stream):
             for i in range(reps + 3):
                 if cold:
                     flush.fill_(i & 0xFF)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream); vocab_once(); b.record(stream)
-                stream.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
-        return statistics.mean(ts)
+                evs.append((a, b))
+        stream.synchronize()
+        return statistics.mean(a.elapsed_time(b) for a, b in evs[3:])
 
     alg_bytes = V * d * 2 + M * d * 2 + M * 4
     t_cold, t_warm = time_vocab(True), time_vocab(False)
