@@ -45,6 +45,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking probe of a barrier phase: returns at once with 1 if the phase has completed, else 0.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
 // Bounded wait.  Returns false (after latching the error) when the phase did not complete in time.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
   for (uint32_t i = 0; i < SPIN_LIMIT; ++i)
@@ -289,24 +301,48 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       if (warp == 0) trace_mark(TR_GEMM + EPI, 3);
     } else if (warp == 1 && lane == 0) {
       // ---- MMA issuer ----
+      // This single thread's instruction latencies add up once per K block, so the loop carries running stage /
+      // parity / descriptor values instead of recomputing them (no integer division, no address rebuilding).
       const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
       bool ok = true;
-      for (int i = 0; i < num_kb && ok; ++i) {
-        const int s = i % stages;
-        const uint32_t round = i / stages;
-        ok = mbar_wait(smem_u32(&bar_full[s]), round & 1, p.status);
-        if (!ok) { abort_flag = 1; break; }
+      int s = 0;
+      uint32_t parity = 0;
+      const uint64_t desc_a0 = make_smem_desc(smem_base);
+      const uint64_t desc_b0 = make_smem_desc(smem_base + A_STAGE_BYTES);
+      const uint64_t desc_step = (uint64_t)(stage_bytes >> 4);     // stage stride in the (address >> 4) field
+      uint64_t desc_a = desc_a0, desc_b = desc_b0;
+      uint32_t bar_f = smem_u32(&bar_full[0]), bar_e = smem_u32(&bar_empty[0]);
+      // A barrier wait costs this thread ~0.14 us even when the phase completed long ago, so after every blocking
+      // wait the remaining stages of the ring round are probed in one batch (their latencies overlap) and the
+      // stages found complete are consumed without waiting again.
+      uint32_t ready_mask = 0;
+      for (int i = 0; i < num_kb; ++i) {
+        if (!((ready_mask >> s) & 1u)) {
+          ok = mbar_wait(bar_f, parity, p.status);
+          if (!ok) { abort_flag = 1; break; }
+          const int left = min(stages - s, num_kb - i);      // stages of this round from s on (s included)
+          uint32_t probe[MAX_STAGES];
+#pragma unroll
+          for (int t = 1; t < MAX_STAGES; ++t) probe[t] = (t < left) ? mbar_test(bar_f + 8 * t, parity) : 0u;
+#pragma unroll
+          for (int t = 1; t < MAX_STAGES; ++t) ready_mask |= probe[t] << ((s + t) & 31);
+        }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = smem_base + s * stage_bytes;
-        const uint64_t desc_a = make_smem_desc(a_addr);
-        const uint64_t desc_b = make_smem_desc(a_addr + A_STAGE_BYTES);
 #pragma unroll
         for (int k4 = 0; k4 < BLOCK_K / UMMA_K; ++k4) {
           // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
           umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (i | k4) != 0 ? 1u : 0u);
         }
         // the stage is handed back to the producers only if a later K block will land in it
-        if (i + stages < num_kb) umma_commit(smem_u32(&bar_empty[s]));
+        if (i + stages < num_kb) umma_commit(bar_e);
+        if (++s == stages) {
+          s = 0; parity ^= 1; ready_mask = 0;
+          desc_a = desc_a0; desc_b = desc_b0;
+          bar_f = smem_u32(&bar_full[0]); bar_e = smem_u32(&bar_empty[0]);
+        } else {
+          desc_a += desc_step; desc_b += desc_step;
+          bar_f += 8; bar_e += 8;
+        }
       }
       if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
     }
