@@ -103,7 +103,10 @@ typedef struct ad_gen_opts {
                             draft_override when that is given); 0 = skip it (needs draft_override) */
   int32_t sync_every;    /* iterations between host checks of the device-side "all rows finished" word;
                             0 = library default (1) */
-  int32_t use_graph;     /* 1 = replay one captured CUDA graph per iteration, 0 = launch kernels directly.
+  int32_t use_graph;     /* 1 = run the loop as a CUDA graph: one launch whose device-side `while` node repeats the
+                            captured iteration until every row has finished (bounded by the longest max_len); if
+                            that graph cannot be built, one graph replay per iteration with host polling.
+                            0 = launch kernels directly.
                             Ignored (direct launches) when the handle was created on the default stream,
                             which cannot be captured. */
 } ad_gen_opts;

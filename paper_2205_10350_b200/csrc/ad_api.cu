@@ -102,10 +102,11 @@ struct ad_handle {
   bool encoded = false;
   int last_vocab_which = -1;
   std::string err;
-  struct GraphEntry { cudaGraphExec_t exec; int launches; };
+  struct GraphEntry { cudaGraphExec_t exec; int launches; bool device_loop; };
   std::map<std::string, GraphEntry> graphs;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
   int launches = 0;          // kernels launched by the last ad_generate (direct) or per graph replay
+  unsigned long long cond_handle = 0;   // non-zero only while the body of a device-side `while` node is captured
 };
 
 namespace {
@@ -311,7 +312,8 @@ int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
 
 // ---- kernel launch helpers -----------------------------------------------------------------------
 
-bool g_use_pdl = true;   // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
+bool g_use_pdl = true;       // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
+bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
 
 // Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
 // themselves wait with griddepcontrol.wait before touching anything a predecessor writes).
@@ -563,7 +565,8 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
   AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   h->launches++;
   AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
-                      pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1)));
+                      pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
+                      auto_commit ? h->cond_handle : 0ull));
   h->last_vocab_which = to_drafts ? 1 : 0;
   return AD_OK;
 }
@@ -673,6 +676,8 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
     return fail(nullptr, AD_ERR_CUDA, "no CUDA device");
+  { const char* e = getenv("AD_NO_PDL"); g_use_pdl = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_NO_DEVLOOP"); g_use_devloop = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();
@@ -882,35 +887,87 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
 
   cudaGraphExec_t exec = nullptr;
   int per_iter_launches = 0;
+  bool device_loop = false;
   if (opts->use_graph && h->stream != nullptr) {   // the legacy default stream cannot be captured
     char key[160];
     snprintf(key, sizeof(key), "B%d m%d k%d o%d v%d d%d", B, opts->mode, opts->k, ovr ? 1 : 0, ovr_len, opts->run_drafter);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
-      cudaGraph_t g = nullptr;
       const int before = h->launches;
-      AD_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
-      const int rc = loop_iteration(h, *opts, ovr, ovr_len);
-      cudaError_t e = cudaStreamEndCapture(h->stream, &g);
-      per_iter_launches = h->launches - before;
-      h->launches = before;
-      if (rc != AD_OK) { if (g) cudaGraphDestroy(g); return rc; }
-      if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph capture: ") + cudaGetErrorString(e));
-      e = cudaGraphInstantiate(&exec, g, 0);
-      cudaGraphDestroy(g);
-      if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
-      h->graphs[key] = ad_handle::GraphEntry{exec, per_iter_launches};
+      // First choice: the whole loop as one graph -- a device-side `while` node whose body is one iteration and
+      // whose condition the accept/commit kernel clears; no host round trip between iterations.
+      if (g_use_devloop) {
+        cudaGraph_t g = nullptr;
+        cudaGraphConditionalHandle ch = 0;
+        bool okb = cudaGraphCreate(&g, 0) == cudaSuccess &&
+                   cudaGraphConditionalHandleCreate(&ch, g, 1, cudaGraphCondAssignDefault) == cudaSuccess;
+        cudaGraphNodeParams np = {cudaGraphNodeTypeConditional};
+        np.conditional.handle = ch;
+        np.conditional.type = cudaGraphCondTypeWhile;
+        np.conditional.size = 1;
+        cudaGraphNode_t node;
+        okb = okb && cudaGraphAddNode(&node, g, nullptr, 0, &np) == cudaSuccess;
+        if (okb) {
+          cudaGraph_t body = np.conditional.phGraph_out[0];
+          okb = cudaStreamBeginCaptureToGraph(h->stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+          if (okb) {
+            h->cond_handle = (unsigned long long)ch;
+            const int rc = loop_iteration(h, *opts, ovr, ovr_len);
+            h->cond_handle = 0;
+            cudaGraph_t dummy = nullptr;
+            const cudaError_t e = cudaStreamEndCapture(h->stream, &dummy);
+            okb = rc == AD_OK && e == cudaSuccess;
+          }
+        }
+        per_iter_launches = h->launches - before;
+        h->launches = before;
+        if (okb) okb = cudaGraphInstantiate(&exec, g, 0) == cudaSuccess;
+        if (g) cudaGraphDestroy(g);
+        if (okb) {
+          h->graphs[key] = ad_handle::GraphEntry{exec, per_iter_launches, true};
+          device_loop = true;
+        } else {
+          exec = nullptr;
+          cudaGetLastError();   // clear; fall back to one replay per iteration
+        }
+      }
+      if (!exec) {
+        cudaGraph_t g = nullptr;
+        AD_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+        const int rc = loop_iteration(h, *opts, ovr, ovr_len);
+        cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+        per_iter_launches = h->launches - before;
+        h->launches = before;
+        if (rc != AD_OK) { if (g) cudaGraphDestroy(g); return rc; }
+        if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+        e = cudaGraphInstantiate(&exec, g, 0);
+        cudaGraphDestroy(g);
+        if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+        h->graphs[key] = ad_handle::GraphEntry{exec, per_iter_launches, false};
+      }
     } else {
       exec = it->second.exec;
       per_iter_launches = it->second.launches;
+      device_loop = it->second.device_loop;
     }
   }
 
+  if (device_loop) {
+    // one launch runs every iteration; the data-independent bound on the iteration count travels in loop_it[3]
+    const int limit = max_iters + 1;
+    AD_CUDA(h, cudaMemcpyAsync(h->st.loop_it + 3, &limit, sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    AD_CUDA(h, cudaGraphLaunch(exec, h->stream));
+    int done = 0;
+    AD_CUDA(h, cudaMemcpyAsync(&done, h->st.loop_it + 2, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
+    AD_CUDA(h, cudaStreamSynchronize(h->stream));
+    h->launches += per_iter_launches * done;
+  }
   const int sync_every = opts->sync_every > 0 ? opts->sync_every : 1;
   int iters = 0;
   volatile int* flag = h->host_flag;
   flag[0] = 0;
-  while (iters < max_iters + sync_every) {
+  while (!device_loop && iters < max_iters + sync_every) {
     for (int s = 0; s < sync_every; ++s, ++iters) {
       if (exec) {
         AD_CUDA(h, cudaGraphLaunch(exec, h->stream));
@@ -923,7 +980,7 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
     AD_CUDA(h, cudaStreamSynchronize(h->stream));
     if (flag[0]) break;
   }
-  AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
+  if (!device_loop) AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
   const int w = out_stride < c.max_tgt ? out_stride : c.max_tgt;
   AD_CUDA(h, cudaMemcpy2DAsync(out, sizeof(int) * out_stride, h->st.out_ids, sizeof(int) * c.max_tgt, sizeof(int) * w, B, from_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(out_len, h->st.len, sizeof(int) * B, from_dev(on_host), h->stream));

@@ -4,6 +4,8 @@
 // planning of the drafter and encoder passes.
 #pragma once
 
+#include <cuda_device_runtime_api.h>
+
 #include "ad_common.cuh"
 
 namespace ad {
@@ -131,6 +133,7 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
     for (int b = 0; b < B; ++b) { s_off[b] = acc; acc += s_k[b]; }
     s_off[B] = acc;
     *plan.M = acc;
+    st.loop_it[1] = 0;   // rows-done counter of the accept kernel: every iteration starts from zero
   }
   __syncthreads();
   for (int b = warp; b < B; b += 8) {
@@ -215,6 +218,7 @@ plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
     for (int b = 0; b < B; ++b) { s_off[b] = acc; acc += st.srclen[b]; }
     *plan.M = acc;
     *st.loop_it = 0;
+    st.loop_it[2] = 0;
     *st.all_fin = 0;
   }
   for (int b = tid; b < B; b += 256) {
@@ -422,11 +426,20 @@ __device__ __forceinline__ void commit_row(const DevState& st, const PassPlan& b
 }
 
 // After every row has been committed: loop counter and the "all rows finished" word.  One thread.
-__device__ __forceinline__ void finish_iteration(const DevState& st, const Dims& dm, bool any_active) {
+// cond != 0: the iteration runs inside a device-side `while` graph node; the node repeats while its condition
+// is non-zero, so it is cleared when every row has finished -- or, as a bound that does not depend on the data,
+// when the iteration counter st.loop_it[2] reaches the limit st.loop_it[3] the host stored before the launch.
+__device__ __forceinline__ void finish_iteration(const DevState& st, const Dims& dm, bool any_active,
+                                                 unsigned long long cond) {
   int all = 1;
   for (int b = 0; b < dm.B; ++b) all &= (__ldcg(st.fin + b) != 0);
   if (any_active) *st.loop_it += 1;
   *st.all_fin = all;
+  if (cond) {
+    const int it = st.loop_it[2] + 1;
+    st.loop_it[2] = it;
+    cudaGraphSetConditional(cond, (all || it >= st.loop_it[3]) ? 0u : 1u);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -444,7 +457,7 @@ __device__ __forceinline__ void finish_iteration(const DevState& st, const Dims&
 __global__ void __launch_bounds__(1024)
 argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
                      const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts, int auto_commit,
-                     unsigned int* done_ctr) {
+                     unsigned int* done_ctr, unsigned long long cond) {
   trace_mark(TR_ACCEPT, 0);
   pdl_launch();
   pdl_wait();
@@ -504,7 +517,7 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
         const unsigned int t = atomicAdd(done_ctr, n > 0 ? 0x10001u : 1u);
         if ((t & 0xffffu) == (unsigned)dm.B - 1) {
           __threadfence();
-          finish_iteration(st, dm, ((t >> 16) + (n > 0 ? 1u : 0u)) != 0);
+          finish_iteration(st, dm, ((t >> 16) + (n > 0 ? 1u : 0u)) != 0, cond);
           *done_ctr = 0;
         }
       }
@@ -535,7 +548,7 @@ commit_kernel(DevState st, PassPlan blk, Dims dm, const int* n_in) {
     if (lane == 0 && nacc > 0) atomicOr(&s_active, 1);
   }
   __syncthreads();
-  if (threadIdx.x == 0) finish_iteration(st, dm, s_active != 0);
+  if (threadIdx.x == 0) finish_iteration(st, dm, s_active != 0, 0ull);
 }
 
 // Teacher-forced commit: the caller supplies the accepted tokens.  grid = 1, block = 256.
