@@ -313,6 +313,7 @@ int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
 // ---- kernel launch helpers -----------------------------------------------------------------------
 
 bool g_use_pdl = true;       // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
+bool g_use_graph_encode = true;   // AD_NO_ENCODE_GRAPH=1: launch the encoder kernels directly
 bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
 
 // Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
@@ -678,6 +679,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
     return fail(nullptr, AD_ERR_CUDA, "no CUDA device");
   { const char* e = getenv("AD_NO_PDL"); g_use_pdl = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_DEVLOOP"); g_use_devloop = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_NO_ENCODE_GRAPH"); g_use_graph_encode = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();
@@ -753,17 +755,49 @@ extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, c
     for (int b = 0; b < B; ++b)
       if (src_len[b] < 1 || src_len[b] > c.max_src || src_len[b] > src_stride)
         return fail(h, src_len[b] > c.max_src ? AD_ERR_CAPACITY : AD_ERR_ARG, "src_len outside 1..min(max_src, src_stride)");
-  if (B != h->B) drop_graphs(h);
+  // (captured graphs are keyed by the batch size, so a different B simply uses other entries)
   h->B = B;
   h->dims.B = B;
   h->encoded = false;
   const int w = src_stride < c.max_src ? src_stride : c.max_src;
   AD_CUDA(h, cudaMemcpy2DAsync(h->st.src, sizeof(int) * c.max_src, src, sizeof(int) * src_stride, sizeof(int) * w, B, to_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, src_len, sizeof(int) * B, to_dev(on_host), h->stream));
-  h->launches++;
-  AD_CUDA(h, launch_k(plan_encode_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_ENCODE].plan, h->dims));
-  AD_TRY(encoder_pass(h, h->ar, true));
-  if (c.has_drafter) AD_TRY(encoder_pass(h, h->nar, false));
+  // The encoder pass reads its inputs from fixed workspace buffers, so on a capturable stream it is captured
+  // once per batch size and replayed (about fifty launches otherwise paid on the host for every sentence).
+  auto enqueue = [&]() -> int {
+    h->launches++;
+    AD_CUDA(h, launch_k(plan_encode_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_ENCODE].plan, h->dims));
+    AD_TRY(encoder_pass(h, h->ar, true));
+    if (c.has_drafter) AD_TRY(encoder_pass(h, h->nar, false));
+    return AD_OK;
+  };
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (h->stream != nullptr) cudaStreamIsCapturing(h->stream, &cap);
+  if (h->stream != nullptr && cap == cudaStreamCaptureStatusNone && g_use_graph_encode) {
+    char key[32];
+    snprintf(key, sizeof(key), "encode B%d", B);
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+      cudaGraph_t g = nullptr;
+      const int before = h->launches;
+      AD_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      const int rc = enqueue();
+      const cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+      const int n = h->launches - before;
+      h->launches = before;
+      if (rc != AD_OK) { if (g) cudaGraphDestroy(g); return rc; }
+      if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("encoder graph capture: ") + cudaGetErrorString(e));
+      cudaGraphExec_t exec = nullptr;
+      const cudaError_t e2 = cudaGraphInstantiate(&exec, g, 0);
+      cudaGraphDestroy(g);
+      if (e2 != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("encoder graph instantiate: ") + cudaGetErrorString(e2));
+      it = h->graphs.emplace(key, ad_handle::GraphEntry{exec, n, false}).first;
+    }
+    AD_CUDA(h, cudaGraphLaunch(it->second.exec, h->stream));
+    h->launches += it->second.launches;
+  } else {
+    AD_TRY(enqueue());
+  }
   h->encoded = true;
   h->last_vocab_which = -1;
   if (on_host) return read_status(h);
