@@ -365,7 +365,7 @@ cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap&
   // the ring doubles as the epilogue's transposition buffer (up to 128 rows of 132 floats)
   const size_t ring = (size_t)stages * (tc::A_STAGE_BYTES + p.ntile * tc::BLOCK_K * 2);
   const size_t smem = std::max(ring, (size_t)std::min(p.ntile, 128) * 132 * sizeof(float)) + 1024;
-  return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(128), smem, st, mw, mx, p, stages);
+  return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(tc::THREADS), smem, st, mw, mx, p, stages);
 }
 
 template <int EPI>
@@ -451,7 +451,13 @@ int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, co
   const size_t stride = (size_t)pc.M_cap * d;
   h->launches++;
   cudaError_t e;
-  if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+  if (pc.M_cap >= 512 && d % 128 == 0 && d <= 1024) {   // many tokens: a warp per token
+    dim3 rgrid((pc.M_cap + 7) / 8);
+    if (h->bf16) e = launch_k(layernorm_rows_kernel<bf16>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+                              (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
+    else e = launch_k(layernorm_rows_kernel<float>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+                      (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
+  } else if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
                             (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
   else e = launch_k(layernorm_kernel<float>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
                     (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
@@ -1110,6 +1116,7 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part_val, const int
   const int m = blockIdx.x, lane = threadIdx.x;
   float v = -INFINITY;
   int idx = 0x7fffffff;
+  pdl_wait();   // the partials come from the kernel before this one
   for (int t = lane; t < n_tiles; t += 32) {
     const float ov = part_val[(size_t)m * n_tiles + t];
     const int oi = part_idx[(size_t)m * n_tiles + t];
@@ -1146,8 +1153,8 @@ extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, in
     return AD_ERR_ARG;
   }
   if (e != cudaSuccess) return AD_ERR_CUDA;
-  argmax_rows_kernel<<<M, 32, 0, st>>>(pv, pi, tiles, M, argmax);
-  return cudaGetLastError() == cudaSuccess ? AD_OK : AD_ERR_CUDA;
+  e = launch_k(argmax_rows_kernel, dim3(M), dim3(32), 0, st, (const float*)pv, (const int*)pi, tiles, M, argmax);
+  return e == cudaSuccess ? AD_OK : AD_ERR_CUDA;
 }
 
 extern "C" int ad_linear(const void* x, const void* W, const float* bias, int32_t dtype, int32_t M, int32_t K,

@@ -83,12 +83,14 @@ __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.laun
 
 // Optional timeline tracing (compile with -DAD_TRACE): thread 0 of CTA (0,0,0) of every kernel stamps the
 // global nanosecond timer at entry (phase 0), after the dependency wait (phase 1), at exit (phase 2) and at
-// kernel-specific points in between (phases 3..7).
+// kernel-specific points in between (phases 3..7); the last CTA along x does the same under id + 16.
 #ifdef AD_TRACE
 __device__ unsigned long long g_trace_buf[1 << 15];
 __device__ unsigned int g_trace_n;
 __device__ __forceinline__ void trace_mark(int id, int phase) {
-  if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+  const bool first = blockIdx.x == 0, last = blockIdx.x == gridDim.x - 1 && gridDim.x > 1;
+  if (threadIdx.x == 0 && (first || last) && blockIdx.y == 0 && blockIdx.z == 0) {
+    if (last) id += 16;
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     const unsigned int i = atomicAdd(&g_trace_n, 1u);

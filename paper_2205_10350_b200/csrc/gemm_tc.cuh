@@ -7,8 +7,10 @@
 // Both operands are K-major (row-major [rows, K]) and land in shared memory in the 128-byte-swizzled
 // canonical layout that the TMA and the MMA shared-memory descriptor agree on.
 //
-// Thread roles inside the 128-thread CTA: lane 0 of warp 0 issues TMA loads, lane 0 of warp 1 issues the
-// MMAs, then all four warps read their 32 TMEM lanes back (tcgen05.ld 32x32b) for the epilogue.
+// Thread roles inside the 256-thread CTA: lane 0 of several warps issues TMA loads, lane 0 of warp 1 issues the
+// MMAs, then all eight warps take part in the epilogue: warp w reads the 32 TMEM lanes of quadrant w % 4
+// (tcgen05.ld 32x32b) and the two warps of a quadrant share its token columns.  The epilogue is a chain of
+// dependent instructions per thread, so halving each thread's share of it shortens the kernel.
 // Every mbarrier wait is bounded; on expiry the kernel latches AD_ERR_TIMEOUT, frees its TMEM and returns.
 #pragma once
 
@@ -19,6 +21,7 @@ namespace tc {
 
 constexpr int BLOCK_N_FEAT = 128;   // weight rows per CTA = MMA M
 constexpr int BLOCK_K = 64;         // bf16 elements per 128-byte swizzle row
+constexpr int THREADS = 256;        // 8 warps: two per tensor-memory lane quadrant
 constexpr int UMMA_K = 16;          // K of one tcgen05.mma kind::f16
 constexpr int A_STAGE_BYTES = BLOCK_N_FEAT * BLOCK_K * 2;   // 16 KiB
 constexpr int MAX_STAGES = 8;
@@ -154,6 +157,62 @@ __device__ __forceinline__ void warp_argmax_lane(float v, float& best, int& lane
   lane_of_best = __ffs(bal) - 1;
 }
 
+// Arg-max over the 32 lanes for 32 values per lane at once.  v[j] is this lane's candidate for item j; on
+// return lane L holds, for item L, the largest candidate and the lowest lane that offered it.  Each halving
+// step sends one half of the items a lane still holds to its partner and keeps the other half, so that every
+// item costs about one exchange instead of five.
+__device__ __forceinline__ void warp_argmax_items(float (&v)[32], int lane, float& best, int& from) {
+  int src[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) src[j] = lane;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const bool up = (lane & o) != 0;                 // this lane keeps the upper half of its items
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float keep_v = up ? v[i + o] : v[i];
+      const int keep_s = up ? src[i + o] : src[i];
+      const float send_v = up ? v[i] : v[i + o];
+      const int send_s = up ? src[i] : src[i + o];
+      const float ov = __shfl_xor_sync(0xffffffffu, send_v, o);
+      const int os = __shfl_xor_sync(0xffffffffu, send_s, o);
+      const bool take = ov > keep_v || (ov == keep_v && os < keep_s);
+      v[i] = take ? ov : keep_v;
+      src[i] = take ? os : keep_s;
+    }
+  }
+  best = v[0];
+  from = src[0];
+}
+// The same for 16 items per lane: lanes 2j and 2j+1 both end up with item j.
+__device__ __forceinline__ void warp_argmax_items16(float (&v)[16], int lane, float& best, int& from) {
+  int src[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) src[j] = lane;
+#pragma unroll
+  for (int o = 16; o > 1; o >>= 1) {
+    const int h = o >> 1;                            // items kept after this step
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < h; ++i) {
+      const float keep_v = up ? v[i + h] : v[i];
+      const int keep_s = up ? src[i + h] : src[i];
+      const float send_v = up ? v[i] : v[i + h];
+      const int send_s = up ? src[i] : src[i + h];
+      const float ov = __shfl_xor_sync(0xffffffffu, send_v, o);
+      const int os = __shfl_xor_sync(0xffffffffu, send_s, o);
+      const bool take = ov > keep_v || (ov == keep_v && os < keep_s);
+      v[i] = take ? ov : keep_v;
+      src[i] = take ? os : keep_s;
+    }
+  }
+  const float ov = __shfl_xor_sync(0xffffffffu, v[0], 1);
+  const int os = __shfl_xor_sync(0xffffffffu, src[0], 1);
+  const bool take = ov > v[0] || (ov == v[0] && os < src[0]);
+  best = take ? ov : v[0];
+  from = take ? os : src[0];
+}
+
 // Best (value, lowest index) over the 32 lanes of a warp.
 __device__ __forceinline__ void warp_argmax(float& v, int& i) {
 #pragma unroll
@@ -188,14 +247,14 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int n, int m
   }
 }
 
-// grid = (ceil(N / 128), ceil(M_cap / ntile), ksplit); block = 128 threads;
+// grid = (ceil(N / 128), ceil(M_cap / ntile), ksplit); block = 256 threads;
 // dynamic smem = stages * stage bytes + 1024.
 //
 // Order of events in a CTA (the part before pdl_wait() overlaps the previous kernel of the stream):
 //   barriers, TMEM allocation, pdl_launch;  producer: weight tiles of the first ring round (token tile 0 only);
 //   pdl_wait;  token count M;  producer: activation tiles, then the rest of the K loop;  MMA issue;  epilogue.
 template <int EPI>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const GemmParams p, const int stages) {
   extern __shared__ uint8_t smem_raw[];
@@ -211,6 +270,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const int t0 = blockIdx.y * ntile;
   const int n0 = blockIdx.x * BLOCK_N_FEAT;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quad = warp & 3, grp = warp >> 2;   // accumulator lane quadrant of this warp; column group in the epilogue
   const int b_stage_bytes = ntile * BLOCK_K * 2;
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
   const int kb_total = p.K / BLOCK_K;
@@ -250,18 +310,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   // never starve it.
   pdl_launch();
 
-  // TMA issue is spread over lane 0 of all four warps: one thread's bulk-tensor copies are processed one after
-  // the other, several threads' copies run side by side.  Stage i of the first ring round belongs to warp i % 4;
+  // TMA issue is spread over lane 0 of all eight warps: one thread's bulk-tensor copies are processed one after
+  // the other, several threads' copies run side by side.  Stage i of the first ring round belongs to warp i;
   // later rounds are fed by warps 0, 2 and 3 (warp 1's lane 0 is busy issuing MMAs).
   if (early && lane == 0) {
     // weights never change: fetch the first ring round before the previous kernel has finished
-    for (int i = warp; i < first_round; i += 4) {
+    for (int i = warp; i < first_round; i += THREADS / 32) {
       const uint32_t bar = smem_u32(&bar_full[i]);
       mbar_expect_tx(bar, (uint32_t)stage_bytes);
       tma_load_2d(smem_base + i * stage_bytes, &map_w, (kb_begin + i) * BLOCK_K, n0, bar);
     }
   }
-  const int n = n0 + warp * 32 + lane;
+  const int n = n0 + quad * 32 + lane;
   const float bias_n = (p.bias && n < p.N) ? p.bias[n] : 0.f;   // a weight as well: no dependency
 
   pdl_wait();
@@ -269,7 +329,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   if (early && lane == 0) {
     // activations of the first ring round (the activation buffer is always valid memory; rows beyond M are
     // simply never stored), issued before the token count is known
-    for (int i = warp; i < first_round; i += 4)
+    for (int i = warp; i < first_round; i += THREADS / 32)
       tma_load_2d(smem_base + i * stage_bytes + A_STAGE_BYTES, &map_x, (kb_begin + i) * BLOCK_K, t0,
                   smem_u32(&bar_full[i]));
   }
@@ -278,9 +338,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   if (valid) {
     if (EPI == EPI_SCATTER) {
-      for (int j = threadIdx.x; j < ntile; j += 128) slot_s[j] = (t0 + j < M) ? p.slot[t0 + j] : 0;
+      for (int j = threadIdx.x; j < ntile; j += THREADS) slot_s[j] = (t0 + j < M) ? p.slot[t0 + j] : 0;
     }
-    if (lane == 0 && warp != 1) {
+    if (lane == 0 && warp != 1 && warp < 4) {
       // ---- TMA producers: everything that was not issued above ----
       // No more producers than stages: a producer's consecutive K blocks are then at most one ring round apart,
       // so its parity wait on an "empty" barrier can never alias a phase two rounds back.
@@ -348,44 +408,73 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     __syncwarp();
 
-    // ---- epilogue: all four warps ----
+    // ---- epilogue: all eight warps ----
     bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
-    ready = __all_sync(0xffffffffu, ready);
+    ready = __syncthreads_and(ready) != 0;     // one verdict for the CTA (also makes slot_s visible)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     trace_mark(TR_GEMM + EPI, 4);
-    if (EPI == EPI_SCATTER) __syncthreads();   // slot_s visible (every thread reaches this point)
-    // The accumulator holds one output feature per thread (TMEM lane) and one token per column.  It is first
-    // transposed through shared memory (the TMA ring is free once the accumulator barrier has fired) into rows
-    // of 128 features per token, so that global stores are 16 bytes per thread and whole 128-feature rows
-    // per warp, and so that the arg-max scan of a token needs no shuffles.
+    // The accumulator holds one output feature per TMEM lane and one token per column.  Warp w reads lanes
+    // 32 (w % 4) .. +31; the two warps of a quadrant take alternate chunks of 16 columns.  The TMA ring is free
+    // once the accumulator barrier has fired and serves as staging memory.
     float* stage = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
-    constexpr int LD = (EPI == EPI_ARGMAX) ? 129 : 132;   // 129: conflict-free column scans; 132: 16-byte aligned rows
+    constexpr int LD = 132;                                // rows stay 16-byte aligned
     const int ntok_all = min(ntile, M - t0);               // valid tokens of this tile (<= 0 only if M == 0)
-    const int sub = ntile < 128 ? ntile : 128;             // tokens transposed per pass (bounds the buffer to 68 KB)
+    const uint32_t tlane = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
+    if (EPI == EPI_ARGMAX) {
+      // No transposition: a warp reduces its 32 features for 16 tokens at a time with a halving exchange, after
+      // which lanes 2j and 2j+1 hold the best of token c + j (lowest id on ties).  The four quadrants' results
+      // meet in shared memory and one thread per token combines them in ascending feature order.
+      float* red_val = stage;                                   // [4][ntile]
+      int* red_idx = reinterpret_cast<int*>(stage + 4 * 256);   // [4][ntile]
+      if (ready) {
+        for (int c = grp * 16; c < ntile && c < ntok_all; c += 32) {
+          float acc[16];
+          tmem_ld16(tlane + static_cast<uint32_t>(c), acc);
+          // columns past the last valid token hold whatever the padded activation rows produced: never stored
+#pragma unroll
+          for (int j = 0; j < 16; ++j) acc[j] = n < p.N ? acc[j] + bias_n : -INFINITY;
+          float my_v;
+          int my_i;
+          warp_argmax_items16(acc, lane, my_v, my_i);
+          const int t = c + (lane >> 1);
+          if (!(lane & 1) && t < ntok_all) {
+            red_val[quad * ntile + t] = my_v;
+            red_idx[quad * ntile + t] = n0 + quad * 32 + my_i;
+          }
+        }
+      }
+      trace_mark(TR_GEMM + EPI, 5);
+      __syncthreads();
+      for (int t = threadIdx.x; t < ntok_all && ready; t += THREADS) {
+        float v = red_val[t];
+        int idx = red_idx[t];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+          const float ov = red_val[w * ntile + t];
+          if (ov > v) { v = ov; idx = red_idx[w * ntile + t]; }
+        }
+        p.part_val[(size_t)(t0 + t) * gridDim.x + blockIdx.x] = v;
+        p.part_idx[(size_t)(t0 + t) * gridDim.x + blockIdx.x] = idx;
+      }
+    }
+    // Other epilogues: the tile is transposed through shared memory into rows of 128 features per token, in
+    // passes of at most 128 tokens (68 KB), so that global stores are 16 bytes per thread and whole rows per warp.
+    const int sub = ntile < 128 ? ntile : 128;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    for (int tb = 0; tb < ntile && tb < ntok_all && ready; tb += sub) {
+    for (int tb = 0; EPI != EPI_ARGMAX && tb < ntile && tb < ntok_all && ready; tb += sub) {
       const int ntok = min(sub, ntok_all - tb);            // valid tokens of this pass
       const int tg = t0 + tb;                              // packed index of the pass's first token
       if (tb > 0) __syncthreads();                         // previous pass has been read out
-      for (int c = 0; c < sub; c += 32) {
-        if (c >= ntok) break;
-        float acc[32];
-        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(tb + c);
-        if (sub - c >= 32) {
-          tmem_ld32(taddr, acc);
-        } else {          // 16-token tile
-          tmem_ld16(taddr, acc);
+      for (int c = grp * 16; c < sub && c < ntok; c += 32) {
+        float acc[16];
+        tmem_ld16(tlane + static_cast<uint32_t>(tb + c), acc);
 #pragma unroll
-          for (int j = 16; j < 32; ++j) acc[j] = 0.f;
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < 16; ++j) {
           if (c + j < ntok) {
             float v = acc[j] + bias_n;
             if (EPI == EPI_ACT && p.relu) v = fmaxf(v, 0.f);
-            if (EPI == EPI_ARGMAX && n >= p.N) v = -INFINITY;
-            stage[(c + j) * LD + threadIdx.x] = v;
+            stage[(c + j) * LD + quad * 32 + lane] = v;
           }
         }
       }
@@ -395,7 +484,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         float* out = p.out_f32 + (size_t)blockIdx.z * p.M_cap * p.N;
         const int col = n0 + lane * 4;
         const bool vec = (p.N & 3) == 0;
-        for (int r = warp; r < ntok; r += 4) {
+        for (int r = warp; r < ntok; r += THREADS / 32) {
           const float4 v = *reinterpret_cast<const float4*>(stage + r * LD + lane * 4);
           float* dst = out + (size_t)(tg + r) * p.N + col;
           if (vec && col + 3 < p.N) {
@@ -419,7 +508,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           base = reinterpret_cast<bf16*>(p.dst[seg]);
         }
         const bool vec = (width & 7) == 0;
-        for (int r = warp * 2 + half; r < ntok; r += 8) {
+        for (int r = warp * 2 + half; r < ntok; r += THREADS / 16) {
           const float* srow = stage + r * LD + f0;
           const float4 a = *reinterpret_cast<const float4*>(srow);
           const float4 b = *reinterpret_cast<const float4*>(srow + 4);
@@ -439,32 +528,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int t = 0; t < 8; ++t)
               if (t < lim) dst[t] = __float2bfloat16_rn(vals[t]);
           }
-        }
-      } else {
-        // EPI_ARGMAX: `parts` threads share a token, each scanning 128 / parts consecutive features in
-        // ascending order (strict > keeps the lowest id); the parts are then combined in ascending order too.
-        const int parts = 128 / sub;
-        const int per = 128 / parts;
-        const int tok = (int)threadIdx.x / parts, part = (int)threadIdx.x % parts;
-        float v = -INFINITY;
-        int idx = 0;
-        if (tok < ntok) {
-          const float* srow = stage + tok * LD + part * per;
-          for (int f = 0; f < per; ++f) {
-            const float x = srow[f];
-            if (x > v) { v = x; idx = f; }
-          }
-          idx += n0 + part * per;
-        }
-        // combine the parts of a token: they sit in consecutive lanes (parts is a power of two <= 8)
-        for (int o = 1; o < parts; o <<= 1) {
-          const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-          if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-        }
-        if (tok < ntok && part == 0) {
-          p.part_val[(size_t)(tg + tok) * gridDim.x + blockIdx.x] = v;
-          p.part_idx[(size_t)(tg + tok) * gridDim.x + blockIdx.x] = idx;
         }
       }
     }

@@ -372,6 +372,76 @@ layernorm_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, i
   trace_mark(TR_LN, 2);
 }
 
+// The same operation for large token counts: one warp per token (no block-wide barrier), 8 tokens per CTA.
+// grid = ceil(M_cap / 8), block = 256, d <= 1024 and a multiple of 128.
+template <typename ActT>
+__global__ void __launch_bounds__(256)
+layernorm_rows_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, int nsplit, size_t split_stride,
+                      const float* __restrict__ bias, const float* resid, const float* __restrict__ g,
+                      const float* __restrict__ bta, int d, float eps, float* y, ActT* __restrict__ yb) {
+  trace_mark(TR_LN, 0);
+  pdl_launch();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int per = d >> 7;                               // float4 groups per lane (d / 128), <= 8
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 cb[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) cb[i] = (i < per && bias) ? reinterpret_cast<const float4*>(bias)[lane + 32 * i] : zero4;
+  pdl_wait();
+  trace_mark(TR_LN, 1);
+  const int m = blockIdx.x * 8 + warp;
+  if (m < *M_ptr) {
+    const size_t row = (size_t)m * (d >> 2);
+    float4 xv[8];
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float4 v = zero4;
+      if (i < per) {
+        const size_t off = row + lane + 32 * i;
+        v = resid ? reinterpret_cast<const float4*>(resid)[off] : zero4;
+        v.x += cb[i].x; v.y += cb[i].y; v.z += cb[i].z; v.w += cb[i].w;
+        for (int sp = 0; sp < nsplit; ++sp) {
+          const float4 q = reinterpret_cast<const float4*>(pre + sp * split_stride)[off];
+          v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+      }
+      xv[i] = v;
+      s += v.x + v.y + v.z + v.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mean = s / (float)d;
+    float vs = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i < per) {
+        const float a = xv[i].x - mean, b = xv[i].y - mean, c = xv[i].z - mean, e = xv[i].w - mean;
+        vs += a * a + b * b + c * c + e * e;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) vs += __shfl_xor_sync(0xffffffffu, vs, o);
+    const float inv = rsqrtf(vs / (float)d + eps);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i < per) {
+        const float4 gv = reinterpret_cast<const float4*>(g)[lane + 32 * i];
+        const float4 bv = reinterpret_cast<const float4*>(bta)[lane + 32 * i];
+        float4 o;
+        o.x = gv.x * ((xv[i].x - mean) * inv) + bv.x;
+        o.y = gv.y * ((xv[i].y - mean) * inv) + bv.y;
+        o.z = gv.z * ((xv[i].z - mean) * inv) + bv.z;
+        o.w = gv.w * ((xv[i].w - mean) * inv) + bv.w;
+        const size_t off = (row + lane + 32 * i) * 4;
+        store4(y + off, o);
+        store4(yb + off, o);
+      }
+    }
+  }
+  trace_mark(TR_LN, 2);
+}
+
 // dst[j, :] = src[gidx[j], :] for j < *M_ptr.  grid = M_cap, block = 128.
 template <typename ActT>
 __global__ void __launch_bounds__(128)
