@@ -12,6 +12,7 @@
 
 #include "ad_common.cuh"
 #include "attention.cuh"
+#include "attention_mma.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "steps.cuh"
@@ -414,19 +415,31 @@ cudaError_t launch_attention(dim3 grid, dim3 block, cudaStream_t st, const AttnP
 }
 
 int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, const void* v, void* out,
-              const int* key_base, const int* nkeys_tok, const int* nkeys_row) {
+              const int* key_base, const int* nkeys_tok, const int* nkeys_row, int max_keys,
+              const float* q_bias = nullptr, int q_nsplit = 0) {
   const ad_model_cfg& c = h->cfg;
   AttnParams p;
   p.q = q; p.k = k; p.v = v; p.out = out;
+  p.q_part = q_nsplit > 0 ? h->pre : nullptr; p.q_bias = q_bias; p.q_nsplit = q_nsplit;
+  p.q_stride = (size_t)pc.M_cap * c.d_model;
   p.seg_off = pc.plan.seg_off; p.seg_len = pc.plan.seg_len;
   p.key_base = key_base; p.nkeys_tok = nkeys_tok; p.nkeys_row = nkeys_row;
   p.d = c.d_model;
   // one query per warp while the grid stays within a couple of waves, eight when there are many queries
   const int dh = c.d_model / c.n_heads;
   const bool many = (long long)h->dims.B * c.n_heads * ((pc.seg_max + 7) / 8) > 3LL * num_sms();
+  p.scale = 1.0f / sqrtf((float)dh);
+  // Tensor-core kernel when there are thousands of queries or rows may hold hundreds of keys (max_keys: the
+  // capacity, known on the host); the FFMA kernel spreads few queries and few keys over more CTAs.
+  if (h->bf16 && dh == 64 && (many || max_keys >= 256)) {
+    p.qchunks = (pc.seg_max + AM_Q - 1) / AM_Q;
+    h->launches++;
+    cudaError_t em = launch_k(attention_mma_kernel, dim3(h->dims.B * p.qchunks, c.n_heads), dim3(128), 0, h->stream, p);
+    if (em != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(em));
+    return AD_OK;
+  }
   const int qpw = many ? 8 : 1;
   p.qchunks = (pc.seg_max + 8 * qpw - 1) / (8 * qpw);
-  p.scale = 1.0f / sqrtf((float)dh);
   dim3 grid(h->dims.B * p.qchunks, c.n_heads);
   const dim3 block(256);
   h->launches++;
@@ -497,7 +510,8 @@ int self_attention_sublayer(ad_handle* h, int pk, const Mat& wqkv, const float* 
   p.bias = bqkv; p.dst[0] = h->qbuf; p.dst[1] = kbuf; p.dst[2] = vbuf; p.seg_width = h->cfg.d_model; p.n_direct = 1;
   p.slot = pc.plan.kv_slot;
   AD_TRY(gemm(h, EPI_SCATTER, wqkv, h->yb, pk, pc.plan.M, pc.M_cap, p));
-  AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, pc.plan.row_nk));
+  AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, pc.plan.row_nk,
+                   pk == PK_VERIFY ? h->dims.max_tgt : pc.seg_max));
   int ns = 1;
   AD_TRY(gemm_to_ln(h, wo, h->abuf, pk, &ns));
   return layernorm(h, pc, ns, bo, lng, lnb);
@@ -527,11 +541,22 @@ int decoder_pass(ad_handle* h, int pk, Model& m) {
     void* kb = pk == PK_VERIFY ? (char*)h->kself + l * self_layer : h->ktmp;
     void* vb = pk == PK_VERIFY ? (char*)h->vself + l * self_layer : h->vtmp;
     AD_TRY(self_attention_sublayer(h, pk, L.wqkv, L.bqkv, L.wo, L.bo, L.ln1g, L.ln1b, kb, vb));
-    GemmParams q = {};
-    q.bias = L.cbq; q.out_act = h->qbuf;
-    AD_TRY(gemm(h, EPI_ACT, L.cq, h->yb, pk, pc.plan.M, pc.M_cap, q));
-    AD_TRY(attention(h, pc, h->qbuf, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
-                     h->st.cross_base, nullptr, h->st.srclen));
+    // Query projection of the cross-attention.  With few tokens a full-K walk per CTA is the slow part of the
+    // projection, so it is split along K and the attention kernel adds the partial sums (and the bias) as it
+    // loads its queries.
+    int qs = h->bf16 && pc.M_cap <= 256 ? pc.ksplit_for(L.cq.N, L.cq.K, pc.tile_for(L.cq.N, num_sms())) : 1;
+    if (qs > 1) {
+      int ns_q = 1;
+      AD_TRY(gemm_to_ln(h, L.cq, h->yb, pk, &ns_q));
+      AD_TRY(attention(h, pc, nullptr, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
+                       h->st.cross_base, nullptr, h->st.srclen, c.max_src, L.cbq, ns_q));
+    } else {
+      GemmParams q = {};
+      q.bias = L.cbq; q.out_act = h->qbuf;
+      AD_TRY(gemm(h, EPI_ACT, L.cq, h->yb, pk, pc.plan.M, pc.M_cap, q));
+      AD_TRY(attention(h, pc, h->qbuf, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
+                       h->st.cross_base, nullptr, h->st.srclen, c.max_src));
+    }
     int ns = 1;
     AD_TRY(gemm_to_ln(h, L.co, h->abuf, pk, &ns));
     AD_TRY(layernorm(h, pc, ns, L.cbo, L.ln2g, L.ln2b));

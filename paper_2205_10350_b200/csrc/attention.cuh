@@ -15,6 +15,12 @@ namespace ad {
 
 struct AttnParams {
   const void* q;         // [M_cap, d]
+  // When q_part is set the queries come straight from the split-K partial sums of their projection instead:
+  // q = round_to_activation_type(sum over q_nsplit partials [M_cap, d], q_stride elements apart, + q_bias).
+  const float* q_part;
+  const float* q_bias;   // [d] or null
+  int q_nsplit;
+  size_t q_stride;
   const void* k;         // [slots, d]
   const void* v;         // [slots, d]
   void* out;             // [M_cap, d]
@@ -101,8 +107,19 @@ attention_kernel(const AttnParams p) {
     if (r < nq) {
       nk[t] = p.nkeys_tok ? min(p.nkeys_tok[m0 + r], row_nk) : row_nk;
 #pragma unroll
-      for (int rr = 0; rr < R; ++rr)
-        qs[r][lane + 32 * rr] = to_f32(q[(size_t)(m0 + r) * d + h * DH + lane + 32 * rr]) * p.scale;
+      for (int rr = 0; rr < R; ++rr) {
+        const int col = h * DH + lane + 32 * rr;
+        const size_t off = (size_t)(m0 + r) * d + col;
+        float qv;
+        if (p.q_part) {
+          qv = p.q_bias ? p.q_bias[col] : 0.f;
+          for (int sp = 0; sp < p.q_nsplit; ++sp) qv += p.q_part[sp * p.q_stride + off];
+          qv = to_f32(from_f32<ActT>(qv));     // the value a stored query would have had
+        } else {
+          qv = to_f32(q[off]);
+        }
+        qs[r][lane + 32 * rr] = qv * p.scale;
+      }
     }
   }
 

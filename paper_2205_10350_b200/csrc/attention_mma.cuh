@@ -1,0 +1,202 @@
+// Attention for many queries on the tensor cores (BF16, head dimension 64).
+//
+// Same operation and masking rules as attention_kernel (attention.cuh); used when a pass has thousands of
+// queries, where the FFMA kernel is bound by its multiply-adds.  The tiles of one (row, head) pair are small
+// (at most 64 queries x 64 keys x 64 dims per step), far below the 128-row atoms of the tcgen05 path and not
+// worth a round trip through tensor memory, so the products run as warp-level m16n8k16 MMAs on register
+// fragments: S = Q K^T, online softmax on the accumulator fragments, P (rounded to BF16) reused in place as
+// the A operand of O += P V, with V read through transposing ldmatrix loads.
+//
+// grid = (B * qchunks, H), qchunks = ceil(longest segment / 64); block = 128 threads = 4 warps x 16 queries.
+#pragma once
+
+#include "attention.cuh"
+
+namespace ad {
+
+constexpr int AM_Q = 64;        // queries per CTA
+constexpr int AM_KT = 64;       // keys per shared-memory tile
+constexpr int AM_LD = 64 + 8;   // padded row length (bf16 elements): rows 144 bytes apart, conflict-free fragments
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+// Two 8x8 BF16 matrices, transposed on the way into registers: lanes 0..7 give the row addresses of the first,
+// lanes 8..15 of the second.
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, const void* row_ptr) {
+  const uint32_t addr = static_cast<uint32_t>(__cvta_generic_to_shared(row_ptr));
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+
+__global__ void __launch_bounds__(128)
+attention_mma_kernel(const AttnParams p) {
+  constexpr int DH = 64;
+  __shared__ __align__(16) bf16 ks[AM_KT][AM_LD];
+  __shared__ __align__(16) bf16 vs[AM_KT][AM_LD];
+
+  trace_mark(TR_ATTN, 0);
+  pdl_launch();
+  pdl_wait();
+  trace_mark(TR_ATTN, 1);
+  const int b = blockIdx.x / p.qchunks;
+  const int chunk = blockIdx.x % p.qchunks;
+  const int h = blockIdx.y;
+  const int seg_len = p.seg_len[b];
+  const int seg_off = p.seg_off[b];
+  const int kbase = p.key_base[b];
+  const int row_nk = p.nkeys_row[b];
+  const int i0 = chunk * AM_Q;
+  if (i0 >= seg_len) return;
+  const int nq = min(AM_Q, seg_len - i0);
+  const int m0 = seg_off + i0;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, tq = lane & 3;           // fragment row (0..7) and column pair (0..3) of this lane
+  const int d = p.d;
+  const bf16* q = reinterpret_cast<const bf16*>(p.q);
+  const bf16* kk = reinterpret_cast<const bf16*>(p.k);
+  const bf16* vv = reinterpret_cast<const bf16*>(p.v);
+
+  // this lane's two queries (fragment rows g and g + 8 of the warp's 16) and their visible-key counts
+  const int r0 = warp * 16 + g, r1 = r0 + 8;
+  int nk0 = 0, nk1 = 0;
+  if (r0 < nq) nk0 = p.nkeys_tok ? min(p.nkeys_tok[m0 + r0], row_nk) : row_nk;
+  if (r1 < nq) nk1 = p.nkeys_tok ? min(p.nkeys_tok[m0 + r1], row_nk) : row_nk;
+  // Q as A fragments of the four 16-wide steps along the head dimension
+  uint32_t qa[DH / 16][4];
+  if (p.q_part) {
+    // queries straight from the split-K partial sums of their projection (+ bias), rounded like stored ones
+#pragma unroll
+    for (int s4 = 0; s4 < DH / 16; ++s4) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = (e & 1) ? r1 : r0;
+        const int c = h * DH + s4 * 16 + tq * 2 + (e >> 1) * 8;
+        float2 acc = make_float2(0.f, 0.f);
+        if (r < nq) {
+          if (p.q_bias) acc = *reinterpret_cast<const float2*>(p.q_bias + c);
+          const float* src = p.q_part + (size_t)(m0 + r) * d + c;
+          for (int sp = 0; sp < p.q_nsplit; ++sp) {
+            const float2 v = *reinterpret_cast<const float2*>(src + sp * p.q_stride);
+            acc.x += v.x; acc.y += v.y;
+          }
+        }
+        qa[s4][e] = pack_bf16(acc.x, acc.y);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int s4 = 0; s4 < DH / 16; ++s4) {
+      const int c = h * DH + s4 * 16 + tq * 2;
+      const bf16* q0 = q + (size_t)(m0 + r0) * d + c;
+      const bf16* q1 = q + (size_t)(m0 + r1) * d + c;
+      qa[s4][0] = r0 < nq ? *reinterpret_cast<const uint32_t*>(q0) : 0u;
+      qa[s4][1] = r1 < nq ? *reinterpret_cast<const uint32_t*>(q1) : 0u;
+      qa[s4][2] = r0 < nq ? *reinterpret_cast<const uint32_t*>(q0 + 8) : 0u;
+      qa[s4][3] = r1 < nq ? *reinterpret_cast<const uint32_t*>(q1 + 8) : 0u;
+    }
+  }
+
+  float o[DH / 8][4];
+#pragma unroll
+  for (int t = 0; t < DH / 8; ++t) { o[t][0] = 0.f; o[t][1] = 0.f; o[t][2] = 0.f; o[t][3] = 0.f; }
+  float mx0 = -INFINITY, mx1 = -INFINITY, den0 = 0.f, den1 = 0.f;   // den: this lane's share of the row sums
+
+  for (int j0 = 0; j0 < row_nk; j0 += AM_KT) {
+    __syncthreads();   // previous tile fully consumed
+#pragma unroll
+    for (int i = 0; i < AM_KT * (DH / 8) / 128; ++i) {
+      const int idx = tid + 128 * i;
+      const int j = idx >> 3, c = (idx & 7) * 8;
+      uint4 ku = make_uint4(0u, 0u, 0u, 0u), vu = ku;      // keys that do not exist read as zeros
+      if (j0 + j < row_nk) {
+        const size_t off = (size_t)(kbase + j0 + j) * d + h * DH + c;
+        ku = *reinterpret_cast<const uint4*>(kk + off);
+        vu = *reinterpret_cast<const uint4*>(vv + off);
+      }
+      *reinterpret_cast<uint4*>(&ks[j][c]) = ku;
+      *reinterpret_cast<uint4*>(&vs[j][c]) = vu;
+    }
+    __syncthreads();
+
+    // S = Q K^T for 16 queries x 64 keys: 8 key groups of 8, 4 steps along the head dimension
+    float s[AM_KT / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < AM_KT / 8; ++nt) {
+      s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
+#pragma unroll
+      for (int s4 = 0; s4 < DH / 16; ++s4) {
+        const bf16* kp = &ks[nt * 8 + g][s4 * 16 + tq * 2];
+        mma_bf16_16816(s[nt], qa[s4], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 8));
+      }
+    }
+    // mask, scale, online softmax; element e of group nt is key j0 + nt * 8 + tq * 2 + (e & 1), query row e >> 1
+    float t0 = -INFINITY, t1 = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < AM_KT / 8; ++nt) {
+      const int j = j0 + nt * 8 + tq * 2;
+      s[nt][0] = (j < nk0) ? s[nt][0] * p.scale : -INFINITY;
+      s[nt][1] = (j + 1 < nk0) ? s[nt][1] * p.scale : -INFINITY;
+      s[nt][2] = (j < nk1) ? s[nt][2] * p.scale : -INFINITY;
+      s[nt][3] = (j + 1 < nk1) ? s[nt][3] * p.scale : -INFINITY;
+      t0 = fmaxf(t0, fmaxf(s[nt][0], s[nt][1]));
+      t1 = fmaxf(t1, fmaxf(s[nt][2], s[nt][3]));
+    }
+    t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 1)); t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 2));
+    t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1)); t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
+    const bool on0 = nk0 > j0, on1 = nk1 > j0;       // otherwise no key of this tile is visible to the query
+    const float m0n = on0 ? fmaxf(mx0, t0) : mx0, m1n = on1 ? fmaxf(mx1, t1) : mx1;
+    const float corr0 = on0 ? expf(mx0 - m0n) : 1.f, corr1 = on1 ? expf(mx1 - m1n) : 1.f;   // exp(-inf) = 0 at first
+    mx0 = m0n; mx1 = m1n;
+    float sum0 = 0.f, sum1 = 0.f;
+    uint32_t pa[AM_KT / 16][4];
+#pragma unroll
+    for (int nt = 0; nt < AM_KT / 8; ++nt) {
+      const float p0 = on0 ? expf(s[nt][0] - m0n) : 0.f, p1 = on0 ? expf(s[nt][1] - m0n) : 0.f;
+      const float p2 = on1 ? expf(s[nt][2] - m1n) : 0.f, p3 = on1 ? expf(s[nt][3] - m1n) : 0.f;
+      sum0 += p0 + p1; sum1 += p2 + p3;
+      // accumulator fragments of two neighbouring key groups are exactly one A fragment of 16 keys
+      pa[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    den0 = den0 * corr0 + sum0;
+    den1 = den1 * corr1 + sum1;
+    // O = O * corr + P V
+#pragma unroll
+    for (int dt = 0; dt < DH / 8; ++dt) {
+      o[dt][0] *= corr0; o[dt][1] *= corr0; o[dt][2] *= corr1; o[dt][3] *= corr1;
+#pragma unroll
+      for (int t = 0; t < AM_KT / 16; ++t) {
+        uint32_t v0, v1;
+        ldmatrix_x2_trans(v0, v1, &vs[t * 16 + (lane & 15)][dt * 8]);
+        mma_bf16_16816(o[dt], pa[t], v0, v1);
+      }
+    }
+  }
+
+  den0 += __shfl_xor_sync(0xffffffffu, den0, 1); den0 += __shfl_xor_sync(0xffffffffu, den0, 2);
+  den1 += __shfl_xor_sync(0xffffffffu, den1, 1); den1 += __shfl_xor_sync(0xffffffffu, den1, 2);
+  bf16* out = reinterpret_cast<bf16*>(p.out);
+  if (r0 < nq && nk0 > 0) {
+    const float inv = 1.f / den0;
+    bf16* dst = out + (size_t)(m0 + r0) * d + h * DH + tq * 2;
+#pragma unroll
+    for (int dt = 0; dt < DH / 8; ++dt) *reinterpret_cast<uint32_t*>(dst + dt * 8) = pack_bf16(o[dt][0] * inv, o[dt][1] * inv);
+  }
+  if (r1 < nq && nk1 > 0) {
+    const float inv = 1.f / den1;
+    bf16* dst = out + (size_t)(m0 + r1) * d + h * DH + tq * 2;
+#pragma unroll
+    for (int dt = 0; dt < DH / 8; ++dt) *reinterpret_cast<uint32_t*>(dst + dt * 8) = pack_bf16(o[dt][2] * inv, o[dt][3] * inv);
+  }
+  trace_mark(TR_ATTN, 2);
+}
+
+}  // namespace ad
