@@ -342,12 +342,12 @@ int num_sms() {
   return n;
 }
 
-// Ring depth: as deep as ~200 KB of shared memory allows when the grid fits one wave; when a small-token GEMM
-// has more CTAs than SMs (the vocabulary projection), half of that so that two CTAs share an SM and the
-// whole grid is resident at once.
+// Ring depth: as deep as ~200 KB of shared memory allows when the grid fits one wave; with more CTAs than SMs,
+// half of that so that two CTAs share an SM: up to twice the SM count the whole grid is then resident at once,
+// beyond that one CTA's prologue and epilogue overlap the other's K loop.
 int tc_stages(int ntile, int kb, int n_ctas) {
   const int stage = tc::A_STAGE_BYTES + ntile * tc::BLOCK_K * 2;
-  const int budget = ((ntile <= 64 && n_ctas > num_sms()) || n_ctas > 2 * num_sms()) ? 100 * 1024 : 200 * 1024;
+  const int budget = n_ctas > num_sms() ? 100 * 1024 : 200 * 1024;
   int s = clampi(budget / stage, 1, tc::MAX_STAGES);
   return s < kb ? s : (kb > 0 ? kb : 1);
 }
@@ -545,7 +545,7 @@ int decoder_pass(ad_handle* h, int pk, Model& m) {
     // projection, so it is split along K and the attention kernel adds the partial sums (and the bias) as it
     // loads its queries.
     int qs = h->bf16 && pc.M_cap <= 256 ? pc.ksplit_for(L.cq.N, L.cq.K, pc.tile_for(L.cq.N, num_sms())) : 1;
-    if (qs > 1) {
+    if (qs > 1 && qs <= ATT_MAX_QSPLIT) {
       int ns_q = 1;
       AD_TRY(gemm_to_ln(h, L.cq, h->yb, pk, &ns_q));
       AD_TRY(attention(h, pc, nullptr, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,

@@ -53,6 +53,7 @@ __device__ __forceinline__ void load8(const float* p, float* out) {
 }
 
 constexpr int ATT_WARPS = 8;   // warps per CTA
+constexpr int ATT_MAX_QSPLIT = 16;   // most split-K partials a query may be summed from
 constexpr int ATT_KT = 64;     // keys per shared-memory tile
 
 template <int DH, int QPW>
@@ -113,7 +114,11 @@ attention_kernel(const AttnParams p) {
         float qv;
         if (p.q_part) {
           qv = p.q_bias ? p.q_bias[col] : 0.f;
-          for (int sp = 0; sp < p.q_nsplit; ++sp) qv += p.q_part[sp * p.q_stride + off];
+          float part[ATT_MAX_QSPLIT];                  // all partials in one round trip
+#pragma unroll
+          for (int sp = 0; sp < ATT_MAX_QSPLIT; ++sp) part[sp] = sp < p.q_nsplit ? p.q_part[sp * p.q_stride + off] : 0.f;
+#pragma unroll
+          for (int sp = 0; sp < ATT_MAX_QSPLIT; ++sp) qv += part[sp];
           qv = to_f32(from_f32<ActT>(qv));     // the value a stored query would have had
         } else {
           qv = to_f32(q[off]);

@@ -19,7 +19,7 @@ constexpr int AM_KT = 64;       // keys per shared-memory tile
 constexpr int AM_LD = 64 + 8;   // padded row length (bf16 elements): rows 144 bytes apart, conflict-free fragments
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
       "{%0, %1, %2, %3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -83,10 +83,12 @@ attention_mma_kernel(const AttnParams p) {
         if (r < nq) {
           if (p.q_bias) acc = *reinterpret_cast<const float2*>(p.q_bias + c);
           const float* src = p.q_part + (size_t)(m0 + r) * d + c;
-          for (int sp = 0; sp < p.q_nsplit; ++sp) {
-            const float2 v = *reinterpret_cast<const float2*>(src + sp * p.q_stride);
-            acc.x += v.x; acc.y += v.y;
-          }
+          float2 part[ATT_MAX_QSPLIT];                 // all partials in one round trip
+#pragma unroll
+          for (int sp = 0; sp < ATT_MAX_QSPLIT; ++sp)
+            part[sp] = sp < p.q_nsplit ? *reinterpret_cast<const float2*>(src + sp * p.q_stride) : make_float2(0.f, 0.f);
+#pragma unroll
+          for (int sp = 0; sp < ATT_MAX_QSPLIT; ++sp) { acc.x += part[sp].x; acc.y += part[sp].y; }
         }
         qa[s4][e] = pack_bf16(acc.x, acc.y);
       }
@@ -109,33 +111,55 @@ attention_mma_kernel(const AttnParams p) {
   for (int t = 0; t < DH / 8; ++t) { o[t][0] = 0.f; o[t][1] = 0.f; o[t][2] = 0.f; o[t][3] = 0.f; }
   float mx0 = -INFINITY, mx1 = -INFINITY, den0 = 0.f, den1 = 0.f;   // den: this lane's share of the row sums
 
+  // K/V tiles travel global -> registers -> shared memory; the loads of tile t + 1 are issued before the
+  // arithmetic of tile t so that their latency is hidden behind it.
+  constexpr int PIECES = AM_KT * (DH / 8) / 128;    // 16-byte pieces per thread, per matrix and tile
+  uint4 kreg[PIECES], vreg[PIECES];
+  auto fetch = [&](int j0) {
+#pragma unroll
+    for (int i = 0; i < PIECES; ++i) {
+      const int idx = tid + 128 * i;
+      const int j = idx >> 3, c = (idx & 7) * 8;
+      kreg[i] = make_uint4(0u, 0u, 0u, 0u);          // keys that do not exist read as zeros
+      vreg[i] = kreg[i];
+      if (j0 + j < row_nk) {
+        const size_t off = (size_t)(kbase + j0 + j) * d + h * DH + c;
+        kreg[i] = *reinterpret_cast<const uint4*>(kk + off);
+        vreg[i] = *reinterpret_cast<const uint4*>(vv + off);
+      }
+    }
+  };
+  fetch(0);
   for (int j0 = 0; j0 < row_nk; j0 += AM_KT) {
     __syncthreads();   // previous tile fully consumed
 #pragma unroll
-    for (int i = 0; i < AM_KT * (DH / 8) / 128; ++i) {
+    for (int i = 0; i < PIECES; ++i) {
       const int idx = tid + 128 * i;
       const int j = idx >> 3, c = (idx & 7) * 8;
-      uint4 ku = make_uint4(0u, 0u, 0u, 0u), vu = ku;      // keys that do not exist read as zeros
-      if (j0 + j < row_nk) {
-        const size_t off = (size_t)(kbase + j0 + j) * d + h * DH + c;
-        ku = *reinterpret_cast<const uint4*>(kk + off);
-        vu = *reinterpret_cast<const uint4*>(vv + off);
-      }
-      *reinterpret_cast<uint4*>(&ks[j][c]) = ku;
-      *reinterpret_cast<uint4*>(&vs[j][c]) = vu;
+      *reinterpret_cast<uint4*>(&ks[j][c]) = kreg[i];
+      *reinterpret_cast<uint4*>(&vs[j][c]) = vreg[i];
     }
     __syncthreads();
+    if (j0 + AM_KT < row_nk) fetch(j0 + AM_KT);
 
+    if (warp * 16 >= nq) continue;                   // none of this warp's queries exists: it only helps loading
     // S = Q K^T for 16 queries x 64 keys: 8 key groups of 8, 4 steps along the head dimension
+    // (the step along the head dimension is the outer loop: consecutive MMAs then go to different accumulators
+    // and do not wait for one another)
     float s[AM_KT / 8][4];
 #pragma unroll
-    for (int nt = 0; nt < AM_KT / 8; ++nt) {
-      s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
+    for (int nt = 0; nt < AM_KT / 8; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
 #pragma unroll
-      for (int s4 = 0; s4 < DH / 16; ++s4) {
+    for (int s4 = 0; s4 < DH / 16; ++s4) {
+      uint32_t kb0[AM_KT / 8], kb1[AM_KT / 8];
+#pragma unroll
+      for (int nt = 0; nt < AM_KT / 8; ++nt) {
         const bf16* kp = &ks[nt * 8 + g][s4 * 16 + tq * 2];
-        mma_bf16_16816(s[nt], qa[s4], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 8));
+        kb0[nt] = *reinterpret_cast<const uint32_t*>(kp);
+        kb1[nt] = *reinterpret_cast<const uint32_t*>(kp + 8);
       }
+#pragma unroll
+      for (int nt = 0; nt < AM_KT / 8; ++nt) mma_bf16_16816(s[nt], qa[s4], kb0[nt], kb1[nt]);
     }
     // mask, scale, online softmax; element e of group nt is key j0 + nt * 8 + tq * 2 + (e & 1), query row e >> 1
     float t0 = -INFINITY, t1 = -INFINITY;
@@ -170,14 +194,14 @@ attention_mma_kernel(const AttnParams p) {
     den1 = den1 * corr1 + sum1;
     // O = O * corr + P V
 #pragma unroll
-    for (int dt = 0; dt < DH / 8; ++dt) {
-      o[dt][0] *= corr0; o[dt][1] *= corr0; o[dt][2] *= corr1; o[dt][3] *= corr1;
+    for (int dt = 0; dt < DH / 8; ++dt) { o[dt][0] *= corr0; o[dt][1] *= corr0; o[dt][2] *= corr1; o[dt][3] *= corr1; }
 #pragma unroll
-      for (int t = 0; t < AM_KT / 16; ++t) {
-        uint32_t v0, v1;
-        ldmatrix_x2_trans(v0, v1, &vs[t * 16 + (lane & 15)][dt * 8]);
-        mma_bf16_16816(o[dt], pa[t], v0, v1);
-      }
+    for (int t = 0; t < AM_KT / 16; ++t) {
+      uint32_t v0[DH / 8], v1[DH / 8];
+#pragma unroll
+      for (int dt = 0; dt < DH / 8; ++dt) ldmatrix_x2_trans(v0[dt], v1[dt], &vs[t * 16 + (lane & 15)][dt * 8]);
+#pragma unroll
+      for (int dt = 0; dt < DH / 8; ++dt) mma_bf16_16816(o[dt], pa[t], v0[dt], v1[dt]);
     }
   }
 
