@@ -432,9 +432,16 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   // Tensor-core kernel when there are thousands of queries or rows may hold hundreds of keys (max_keys: the
   // capacity, known on the host); the FFMA kernel spreads few queries and few keys over more CTAs.
   if (h->bf16 && dh == 64 && (many || max_keys >= 256)) {
-    p.qchunks = (pc.seg_max + AM_Q - 1) / AM_Q;
+    // rows with few queries: warps share a 16-query tile and split the keys (2 or 4 key groups)
+    const int ng = pc.seg_max <= 16 ? 4 : (pc.seg_max <= 32 ? 2 : 1);
+    const int qcta = AM_Q / ng;
+    p.qchunks = (pc.seg_max + qcta - 1) / qcta;
     h->launches++;
-    cudaError_t em = launch_k(attention_mma_kernel, dim3(h->dims.B * p.qchunks, c.n_heads), dim3(128), 0, h->stream, p);
+    const dim3 mgrid(h->dims.B * p.qchunks, c.n_heads);
+    cudaError_t em;
+    if (ng == 4) em = launch_k(attention_mma_kernel<4>, mgrid, dim3(128), 0, h->stream, p);
+    else if (ng == 2) em = launch_k(attention_mma_kernel<2>, mgrid, dim3(128), 0, h->stream, p);
+    else em = launch_k(attention_mma_kernel<1>, mgrid, dim3(128), 0, h->stream, p);
     if (em != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(em));
     return AD_OK;
   }

@@ -7,14 +7,14 @@
 // fragments: S = Q K^T, online softmax on the accumulator fragments, P (rounded to BF16) reused in place as
 // the A operand of O += P V, with V read through transposing ldmatrix loads.
 //
-// grid = (B * qchunks, H), qchunks = ceil(longest segment / 64); block = 128 threads = 4 warps x 16 queries.
+// grid = (B * qchunks, H), qchunks = ceil(longest segment / queries per CTA); block = 128 threads.
 #pragma once
 
 #include "attention.cuh"
 
 namespace ad {
 
-constexpr int AM_Q = 64;        // queries per CTA
+constexpr int AM_Q = 64;        // queries per CTA with one key group
 constexpr int AM_KT = 64;       // keys per shared-memory tile
 constexpr int AM_LD = 64 + 8;   // padded row length (bf16 elements): rows 144 bytes apart, conflict-free fragments
 
@@ -36,11 +36,18 @@ __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, co
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
 }
 
+// NG = number of key groups.  With NG = 1 the CTA's four warps take 16 queries each (64 queries per CTA).  When
+// rows have few queries, NG = 2 or 4 warps share a 16-query tile instead (32 or 16 queries per CTA) and split
+// the keys of every K/V tile between them; their running maxima, sums and outputs are merged at the end.
+template <int NG>
 __global__ void __launch_bounds__(128)
 attention_mma_kernel(const AttnParams p) {
   constexpr int DH = 64;
-  __shared__ __align__(16) bf16 ks[AM_KT][AM_LD];
-  __shared__ __align__(16) bf16 vs[AM_KT][AM_LD];
+  constexpr int QT = 4 / NG;            // 16-query tiles per CTA
+  constexpr int KS = AM_KT / NG;        // keys of a tile that one warp handles
+  __shared__ __align__(16) bf16 kv[2][AM_KT][AM_LD];
+  bf16 (*ks)[AM_LD] = kv[0];
+  bf16 (*vs)[AM_LD] = kv[1];
 
   trace_mark(TR_ATTN, 0);
   pdl_launch();
@@ -53,19 +60,22 @@ attention_mma_kernel(const AttnParams p) {
   const int seg_off = p.seg_off[b];
   const int kbase = p.key_base[b];
   const int row_nk = p.nkeys_row[b];
-  const int i0 = chunk * AM_Q;
+  const int i0 = chunk * (16 * QT);
   if (i0 >= seg_len) return;
-  const int nq = min(AM_Q, seg_len - i0);
+  const int nq = min(16 * QT, seg_len - i0);
   const int m0 = seg_off + i0;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tq = lane & 3;           // fragment row (0..7) and column pair (0..3) of this lane
+  const int qtile = warp % QT, grp = warp / QT;     // this warp's query tile and key group
+  const int kofs = grp * KS;                        // first key of a tile that this warp handles
+  const bool active = qtile * 16 < nq;              // otherwise the warp only helps loading
   const int d = p.d;
   const bf16* q = reinterpret_cast<const bf16*>(p.q);
   const bf16* kk = reinterpret_cast<const bf16*>(p.k);
   const bf16* vv = reinterpret_cast<const bf16*>(p.v);
 
   // this lane's two queries (fragment rows g and g + 8 of the warp's 16) and their visible-key counts
-  const int r0 = warp * 16 + g, r1 = r0 + 8;
+  const int r0 = qtile * 16 + g, r1 = r0 + 8;
   int nk0 = 0, nk1 = 0;
   if (r0 < nq) nk0 = p.nkeys_tok ? min(p.nkeys_tok[m0 + r0], row_nk) : row_nk;
   if (r1 < nq) nk1 = p.nkeys_tok ? min(p.nkeys_tok[m0 + r1], row_nk) : row_nk;
@@ -141,31 +151,32 @@ attention_mma_kernel(const AttnParams p) {
     }
     __syncthreads();
     if (j0 + AM_KT < row_nk) fetch(j0 + AM_KT);
+    const int jw = j0 + kofs;                        // first key of this warp's share of the tile
+    if (!active || jw >= row_nk) continue;
 
-    if (warp * 16 >= nq) continue;                   // none of this warp's queries exists: it only helps loading
-    // S = Q K^T for 16 queries x 64 keys: 8 key groups of 8, 4 steps along the head dimension
+    // S = Q K^T for 16 queries x KS keys: KS / 8 key groups of 8, 4 steps along the head dimension
     // (the step along the head dimension is the outer loop: consecutive MMAs then go to different accumulators
     // and do not wait for one another)
-    float s[AM_KT / 8][4];
+    float s[KS / 8][4];
 #pragma unroll
-    for (int nt = 0; nt < AM_KT / 8; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
+    for (int nt = 0; nt < KS / 8; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
 #pragma unroll
     for (int s4 = 0; s4 < DH / 16; ++s4) {
-      uint32_t kb0[AM_KT / 8], kb1[AM_KT / 8];
+      uint32_t kb0[KS / 8], kb1[KS / 8];
 #pragma unroll
-      for (int nt = 0; nt < AM_KT / 8; ++nt) {
-        const bf16* kp = &ks[nt * 8 + g][s4 * 16 + tq * 2];
+      for (int nt = 0; nt < KS / 8; ++nt) {
+        const bf16* kp = &ks[kofs + nt * 8 + g][s4 * 16 + tq * 2];
         kb0[nt] = *reinterpret_cast<const uint32_t*>(kp);
         kb1[nt] = *reinterpret_cast<const uint32_t*>(kp + 8);
       }
 #pragma unroll
-      for (int nt = 0; nt < AM_KT / 8; ++nt) mma_bf16_16816(s[nt], qa[s4], kb0[nt], kb1[nt]);
+      for (int nt = 0; nt < KS / 8; ++nt) mma_bf16_16816(s[nt], qa[s4], kb0[nt], kb1[nt]);
     }
-    // mask, scale, online softmax; element e of group nt is key j0 + nt * 8 + tq * 2 + (e & 1), query row e >> 1
+    // mask, scale, online softmax; element e of group nt is key jw + nt * 8 + tq * 2 + (e & 1), query row e >> 1
     float t0 = -INFINITY, t1 = -INFINITY;
 #pragma unroll
-    for (int nt = 0; nt < AM_KT / 8; ++nt) {
-      const int j = j0 + nt * 8 + tq * 2;
+    for (int nt = 0; nt < KS / 8; ++nt) {
+      const int j = jw + nt * 8 + tq * 2;
       s[nt][0] = (j < nk0) ? s[nt][0] * p.scale : -INFINITY;
       s[nt][1] = (j + 1 < nk0) ? s[nt][1] * p.scale : -INFINITY;
       s[nt][2] = (j < nk1) ? s[nt][2] * p.scale : -INFINITY;
@@ -175,16 +186,16 @@ attention_mma_kernel(const AttnParams p) {
     }
     t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 1)); t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 2));
     t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1)); t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
-    const bool on0 = nk0 > j0, on1 = nk1 > j0;       // otherwise no key of this tile is visible to the query
+    const bool on0 = nk0 > jw, on1 = nk1 > jw;       // otherwise none of these keys is visible to the query
     const float m0n = on0 ? fmaxf(mx0, t0) : mx0, m1n = on1 ? fmaxf(mx1, t1) : mx1;
-    const float corr0 = on0 ? expf(mx0 - m0n) : 1.f, corr1 = on1 ? expf(mx1 - m1n) : 1.f;   // exp(-inf) = 0 at first
+    const float corr0 = on0 ? __expf(mx0 - m0n) : 1.f, corr1 = on1 ? __expf(mx1 - m1n) : 1.f;   // exp(-inf) = 0 at first
     mx0 = m0n; mx1 = m1n;
     float sum0 = 0.f, sum1 = 0.f;
-    uint32_t pa[AM_KT / 16][4];
+    uint32_t pa[KS / 16][4];
 #pragma unroll
-    for (int nt = 0; nt < AM_KT / 8; ++nt) {
-      const float p0 = on0 ? expf(s[nt][0] - m0n) : 0.f, p1 = on0 ? expf(s[nt][1] - m0n) : 0.f;
-      const float p2 = on1 ? expf(s[nt][2] - m1n) : 0.f, p3 = on1 ? expf(s[nt][3] - m1n) : 0.f;
+    for (int nt = 0; nt < KS / 8; ++nt) {
+      const float p0 = on0 ? __expf(s[nt][0] - m0n) : 0.f, p1 = on0 ? __expf(s[nt][1] - m0n) : 0.f;
+      const float p2 = on1 ? __expf(s[nt][2] - m1n) : 0.f, p3 = on1 ? __expf(s[nt][3] - m1n) : 0.f;
       sum0 += p0 + p1; sum1 += p2 + p3;
       // accumulator fragments of two neighbouring key groups are exactly one A fragment of 16 keys
       pa[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
@@ -196,10 +207,10 @@ attention_mma_kernel(const AttnParams p) {
 #pragma unroll
     for (int dt = 0; dt < DH / 8; ++dt) { o[dt][0] *= corr0; o[dt][1] *= corr0; o[dt][2] *= corr1; o[dt][3] *= corr1; }
 #pragma unroll
-    for (int t = 0; t < AM_KT / 16; ++t) {
+    for (int t = 0; t < KS / 16; ++t) {
       uint32_t v0[DH / 8], v1[DH / 8];
 #pragma unroll
-      for (int dt = 0; dt < DH / 8; ++dt) ldmatrix_x2_trans(v0[dt], v1[dt], &vs[t * 16 + (lane & 15)][dt * 8]);
+      for (int dt = 0; dt < DH / 8; ++dt) ldmatrix_x2_trans(v0[dt], v1[dt], &vs[kofs + t * 16 + (lane & 15)][dt * 8]);
 #pragma unroll
       for (int dt = 0; dt < DH / 8; ++dt) mma_bf16_16816(o[dt], pa[t], v0[dt], v1[dt]);
     }
@@ -207,6 +218,42 @@ attention_mma_kernel(const AttnParams p) {
 
   den0 += __shfl_xor_sync(0xffffffffu, den0, 1); den0 += __shfl_xor_sync(0xffffffffu, den0, 2);
   den1 += __shfl_xor_sync(0xffffffffu, den1, 1); den1 += __shfl_xor_sync(0xffffffffu, den1, 2);
+  if (NG > 1) {
+    // Merge the key groups of a query tile.  Every lane of a group > 0 leaves its fragment (32 outputs, two
+    // maxima, two sums) in the tile memory, value-major so that lanes hit different banks; the lane with the
+    // same number in group 0 folds them in.
+    float* rec = reinterpret_cast<float*>(&kv[0][0][0]);   // [36][128]
+    __syncthreads();                                       // all tile reads are done
+    if (grp > 0) {
+#pragma unroll
+      for (int dt = 0; dt < DH / 8; ++dt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) rec[(dt * 4 + e) * 128 + tid] = o[dt][e];
+      rec[32 * 128 + tid] = mx0; rec[33 * 128 + tid] = mx1;
+      rec[34 * 128 + tid] = den0; rec[35 * 128 + tid] = den1;
+    }
+    __syncthreads();
+    if (grp > 0) return;
+#pragma unroll
+    for (int g2 = 1; g2 < NG; ++g2) {
+      const int src = (g2 * QT + qtile) * 32 + lane;       // same query tile, same lane, key group g2
+      const float om0 = rec[32 * 128 + src], om1 = rec[33 * 128 + src];
+      const float n0 = fmaxf(mx0, om0), n1 = fmaxf(mx1, om1);
+      // a row that saw no key at all keeps maximum -inf on both sides: factors 0, nothing to add
+      const float a0 = n0 == -INFINITY ? 0.f : __expf(mx0 - n0), b0 = n0 == -INFINITY ? 0.f : __expf(om0 - n0);
+      const float a1 = n1 == -INFINITY ? 0.f : __expf(mx1 - n1), b1 = n1 == -INFINITY ? 0.f : __expf(om1 - n1);
+      den0 = den0 * a0 + rec[34 * 128 + src] * b0;
+      den1 = den1 * a1 + rec[35 * 128 + src] * b1;
+#pragma unroll
+      for (int dt = 0; dt < DH / 8; ++dt) {
+        o[dt][0] = o[dt][0] * a0 + rec[(dt * 4 + 0) * 128 + src] * b0;
+        o[dt][1] = o[dt][1] * a0 + rec[(dt * 4 + 1) * 128 + src] * b0;
+        o[dt][2] = o[dt][2] * a1 + rec[(dt * 4 + 2) * 128 + src] * b1;
+        o[dt][3] = o[dt][3] * a1 + rec[(dt * 4 + 3) * 128 + src] * b1;
+      }
+      mx0 = n0; mx1 = n1;
+    }
+  }
   bf16* out = reinterpret_cast<bf16*>(p.out);
   if (r0 < nq && nk0 > 0) {
     const float inv = 1.f / den0;

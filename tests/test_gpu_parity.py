@@ -236,3 +236,24 @@ def test_workload5_base_long_source_batch8(base_weights):
     assert all(1 <= len(o) <= 12 for o in outs)
     for b in range(2):
         P.check_free_run(outs[b][:8], g8[b][0][:len(outs[b][:8])], g8[b][1], f"row {b}")
+
+
+def test_long_source_short_blocks(base_weights):
+    """Few queries per row against hundreds of source keys: the attention variant in which the warps of a CTA
+    split the keys of a row and merge their partial softmax results (blocks of at most 12 and of at most 30)."""
+    r = np.random.default_rng(synth.MASTER_SEED + 77)
+    B, S = 2, 300
+    src = r.integers(4, synth.BASE.vocab, size=(B, S)).astype(np.int32)
+    lens = np.array([S, 211], np.int32)
+    src[1, 211:] = synth.PAD
+    om = O.Model(synth.BASE, base_weights, max_pos=S + 1)
+    states = [om.state(src[b, : lens[b]], cap=40) for b in range(B)]
+    g = [st.greedy(10) for st in states]
+    for kmax in (12, 30):
+        dec = binding.AggressiveDecoder(synth.BASE, base_weights, max_batch=B, max_src=S, max_tgt=40, kmax=kmax)
+        streams = np.full((B, 40), 11, np.int32)
+        for b in range(B):
+            streams[b, : len(g[b][0])] = g[b][0]
+            streams[b, 6] = 13
+        tot = P.lockstep(dec, om, src, lens, list(streams), kmax, [40, 40], TOL_BF16, max_steps=2)
+        assert tot["steps"] == 2
