@@ -408,6 +408,52 @@ void orc_top2(const real* logits, int V, int* id1, real* v1, int* id2, real* v2)
   if (v2) *v2 = b >= 0 ? logits[b] : -INFINITY;
 }
 
+/* Relaxed verification of Section 3.2.3 (GAD++) on the scores of one position.  The drafted token is kept
+ * when both conditions of the section hold, otherwise the greedy choice of Eq. 7 is taken:
+ *   Eq. 8:  log P(draft) >= log P(beta-th ranked token)
+ *   Eq. 9:  log P(top-1) - log P(draft) <= tau
+ * log P = score - log(sum of exp(scores)); the normaliser is the same for every token of the position, so both
+ * conditions are evaluated on the scores themselves.  beta >= 1; a negative draft (sentinel) never qualifies.
+ * Outputs (each optional): met = 1 when the draft was kept; top_margin = top-1 minus top-2 score;
+ * decision_margin = how far the scores are from flipping either condition: min(|score(draft) - u_beta|,
+ * |tau - (top1 - score(draft))|), u_beta being the beta-th largest score among the OTHER tokens (the draft passes
+ * Eq. 8 exactly when its score is >= u_beta); +inf where there is nothing to decide. */
+static int cmp_desc(const void* a, const void* b) {
+  const real x = *(const real*)a, y = *(const real*)b;
+  return (x < y) - (x > y);
+}
+int orc_relaxed_choice(const real* logits, int V, int draft, int beta, double tau, int* met, real* top_margin,
+                       real* decision_margin) {
+  int top, second; real v1, v2;
+  orc_top2(logits, V, &top, &v1, &second, &v2);
+  if (top_margin) *top_margin = v1 - v2;
+  if (met) *met = 0;
+  if (decision_margin) *decision_margin = INFINITY;
+  if (draft < 0 || draft >= V || beta < 1) return top;
+  real* sorted = malloc(sizeof(real) * (size_t)V);
+  memcpy(sorted, logits, sizeof(real) * (size_t)V);
+  qsort(sorted, (size_t)V, sizeof(real), cmp_desc);
+  const real vd = logits[draft];
+  const real ranked = sorted[(beta <= V ? beta : V) - 1];          /* score of the beta-th ranked token */
+  const int in_top_beta = vd >= ranked;                            /* Eq. 8 */
+  const int within_tau = (double)v1 - (double)vd <= tau;           /* Eq. 9 */
+  if (decision_margin) {
+    /* beta-th largest among the other tokens: drop one occurrence of the draft's own score from the ranking */
+    real u = -INFINITY;
+    int seen = 0, skipped = 0;
+    for (int i = 0; i < V && seen < beta; ++i) {
+      if (!skipped && sorted[i] == vd) { skipped = 1; continue; }
+      u = sorted[i]; ++seen;
+    }
+    const real m_rank = seen < beta ? INFINITY : (real)fabs((double)vd - (double)u);
+    const real m_tau = (real)fabs(tau - ((double)v1 - (double)vd));
+    *decision_margin = m_rank < m_tau ? m_rank : m_tau;
+  }
+  free(sorted);
+  if (in_top_beta && within_tau) { if (met) *met = 1; return draft; }
+  return top;
+}
+
 /* Acceptance rule.  pred[0..k-1] are the verifier's greedy choices, draft[0..k-1] the drafted tokens
  * they are compared with (draft[i] < 0 is a sentinel that matches nothing).
  *   c = first i with pred[i] != draft[i]  ->  n = c + 1   (the bifurcation token is accepted)
@@ -462,6 +508,29 @@ int orc_verify_block(orc_state* s, int last, const int* draft, int k, int* pred,
       orc_top2(lg + (size_t)i * V, V, &pred[i], &v1, &i2, &v2);
       if (margin) margin[i] = v1 - v2;
     }
+    rc = orc_accept(pred, draft, k, s->m->cfg.eos, finished);
+  }
+  free(tok);
+  if (!logits_out) free(lg);
+  return rc;
+}
+
+/* The same call with the relaxed verification of Section 3.2.3: pred[i] is the drafted token where it meets
+ * the top-beta / tau requirement and the greedy choice elsewhere; the acceptance rule is unchanged (the first
+ * position whose verified token differs from the draft is the bifurcation).  met [k], margin [k] (top-1 minus
+ * top-2), dmargin [k] (see orc_relaxed_choice) are optional. */
+int orc_verify_block_pp(orc_state* s, int last, const int* draft, int k, int beta, double tau, int* pred, int* met,
+                        real* margin, real* dmargin, real* logits_out, int* finished) {
+  int V = s->m->cfg.vocab;
+  int* tok = malloc(sizeof(int) * (size_t)k);
+  real* lg = logits_out ? logits_out : malloc(sizeof(real) * (size_t)k * V);
+  tok[0] = last;
+  for (int i = 1; i < k; ++i) tok[i] = draft[i - 1] >= 0 ? draft[i - 1] : s->m->cfg.pad;
+  int rc = orc_decode_block(s, tok, k, lg);
+  if (rc == 0) {
+    for (int i = 0; i < k; ++i)
+      pred[i] = orc_relaxed_choice(lg + (size_t)i * V, V, draft[i], beta, tau, met ? &met[i] : NULL,
+                                   margin ? &margin[i] : NULL, dmargin ? &dmargin[i] : NULL);
     rc = orc_accept(pred, draft, k, s->m->cfg.eos, finished);
   }
   free(tok);
@@ -612,6 +681,37 @@ int orc_gad(orc_state* s, const orc_model* nar, const real* nar_mem, const int* 
     if (nar) orc_nar_draft(nar, nar_mem, s->S, o, j, k, draft, NULL);
     if (override) for (int t = 0; t < k; ++t) draft[t] = override[j + t];
     int n = orc_verify_block(s, o[j], draft, k, pred, NULL, NULL, &fin);
+    if (n < 1) break;
+    for (int t = 0; t < n; ++t) { o[j + 1 + t] = pred[t]; out[j + t] = pred[t]; }
+    if (tr) {
+      if (tr->it_k) tr->it_k[tr->iterations] = k;
+      if (tr->it_n) tr->it_n[tr->iterations] = n;
+      tr->iterations++; tr->offered += k;
+    }
+    j += n;
+    s->len = j;
+  }
+  free(o); free(draft); free(pred);
+  return j;
+}
+
+/* Generalized mode with the relaxed verification (Section 3.2.3): the loop of orc_gad with
+ * orc_verify_block_pp in place of the exact-match verification. */
+int orc_gad_pp(orc_state* s, const orc_model* nar, const real* nar_mem, const int* override, int kmax,
+               int max_len, int beta, double tau, int* out, orc_trace* tr) {
+  const orc_cfg* c = &s->m->cfg;
+  int* o = malloc(sizeof(int) * (size_t)(max_len + 1));
+  int* draft = malloc(sizeof(int) * (size_t)kmax);
+  int* pred = malloc(sizeof(int) * (size_t)kmax);
+  o[0] = c->bos;
+  int j = 0, fin = 0;
+  s->len = 0;
+  if (tr) { tr->iterations = 0; tr->offered = 0; }
+  while (!fin && j < max_len) {
+    int k = kmax < max_len - j ? kmax : max_len - j;
+    if (nar) orc_nar_draft(nar, nar_mem, s->S, o, j, k, draft, NULL);
+    if (override) for (int t = 0; t < k; ++t) draft[t] = override[j + t];
+    int n = orc_verify_block_pp(s, o[j], draft, k, beta, tau, pred, NULL, NULL, NULL, NULL, &fin);
     if (n < 1) break;
     for (int t = 0; t < n; ++t) { o[j + 1 + t] = pred[t]; out[j + t] = pred[t]; }
     if (tr) {

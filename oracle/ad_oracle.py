@@ -69,6 +69,9 @@ def _lib(real: str):
             "orc_accept": (C.c_int, [ip, ip, C.c_int, C.c_int, ip]),
             "orc_suffix_match": (C.c_int, [ip, C.c_int, ip, C.c_int]),
             "orc_verify_block": (C.c_int, [vp, C.c_int, ip, C.c_int, ip, rp, rp, ip]),
+            "orc_relaxed_choice": (C.c_int, [rp, C.c_int, C.c_int, C.c_int, C.c_double, ip, rp, rp]),
+            "orc_verify_block_pp": (C.c_int, [vp, C.c_int, ip, C.c_int, C.c_int, C.c_double, ip, ip, rp, rp, rp, ip]),
+            "orc_gad_pp": (C.c_int, [vp, vp, rp, ip, C.c_int, C.c_int, C.c_int, C.c_double, ip, C.POINTER(_Trace)]),
             "orc_commit": (None, [vp, C.c_int]),
             "orc_greedy": (C.c_int, [vp, C.c_int, ip, rp]),
             "orc_draft_verify_stream": (C.c_int, [vp, ip, C.c_int, C.c_int, ip, C.POINTER(_Trace)]),
@@ -155,6 +158,15 @@ class Ops:
         self.lib.orc_top2(lg.ctypes.data, lg.shape[0], C.byref(i1), v[0:].ctypes.data, C.byref(i2),
                           v[1:].ctypes.data)
         return i1.value, float(v[0]), i2.value, float(v[1])
+
+    def relaxed_choice(self, logits, draft, beta, tau):
+        """Section 3.2.3 on one position's scores: (verified token, met, top-1 margin, decision margin)."""
+        lg = self._a(logits).ravel()
+        met = C.c_int()
+        tm, dm = np.zeros(1, self.dt), np.zeros(1, self.dt)
+        tok = self.lib.orc_relaxed_choice(lg.ctypes.data, lg.shape[0], int(draft), int(beta), float(tau),
+                                          C.byref(met), tm.ctypes.data, dm.ctypes.data)
+        return tok, bool(met.value), float(tm[0]), float(dm[0])
 
     def accept(self, pred, draft, eos=2):
         p, d = _i32(pred), _i32(draft)
@@ -294,6 +306,25 @@ class State:
             r["logits"] = lg
         return r
 
+    def verify_block_pp(self, last, draft, beta, tau, want_logits=False):
+        """Verification with the relaxed top-beta / tau requirement of Section 3.2.3.
+        Returns dict(pred, met, margin, dmargin, n, finished[, logits]); does not commit."""
+        d = _i32(draft)
+        k = len(d)
+        pred, met = np.empty(k, np.int32), np.empty(k, np.int32)
+        margin, dmargin = np.empty(k, self.m.dt), np.empty(k, self.m.dt)
+        lg = np.empty((k, self.m.V), self.m.dt) if want_logits else None
+        fin = C.c_int()
+        n = self.lib.orc_verify_block_pp(self.h, int(last), _ip(d), k, int(beta), float(tau), _ip(pred), _ip(met),
+                                         margin.ctypes.data, dmargin.ctypes.data,
+                                         lg.ctypes.data if lg is not None else None, C.byref(fin))
+        if n < 1:
+            raise ValueError("verify failed (block does not fit)")
+        r = dict(pred=pred, met=met.astype(bool), margin=margin, dmargin=dmargin, n=n, finished=bool(fin.value))
+        if want_logits:
+            r["logits"] = lg
+        return r
+
     def commit(self, n):
         self.lib.orc_commit(self.h, int(n))
 
@@ -336,4 +367,18 @@ class State:
         n = self.lib.orc_gad(self.h, nar_model.h if nar_model is not None else None,
                              mem.ctypes.data if mem is not None else None,
                              _ip(ov) if ov is not None else None, kmax, max_len, _ip(out), C.byref(tr))
+        return out[:n].copy(), self._trace_out(tr, itk, itn)
+
+    def gad_pp(self, nar_model, kmax, max_len, beta, tau, override=None):
+        """Generalized mode with the relaxed verification of Section 3.2.3."""
+        out = np.empty(max_len, np.int32)
+        tr, itk, itn = self._trace(max_len)
+        mem = nar_model.encode_memory(self.src) if nar_model is not None else None
+        ov = None
+        if override is not None:
+            ov = _i32(np.concatenate([np.asarray(override, np.int32), np.full(kmax + 1, self.m.pad, np.int32)]))
+        n = self.lib.orc_gad_pp(self.h, nar_model.h if nar_model is not None else None,
+                                mem.ctypes.data if mem is not None else None,
+                                _ip(ov) if ov is not None else None, kmax, max_len, int(beta), float(tau),
+                                _ip(out), C.byref(tr))
         return out[:n].copy(), self._trace_out(tr, itk, itn)
