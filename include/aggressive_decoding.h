@@ -194,6 +194,18 @@ int ad_draft_block(ad_handle* h, int32_t k_cap, int32_t* drafts, int32_t* k, int
  * Synchronises; returns a latched device error if there is one (and clears it). */
 int ad_get_state(ad_handle* h, int32_t* len, int32_t* last_tok, int32_t* finished);
 
+/* Relaxed verification (Section 3.2.3, "GAD++", Eq. 8 and Eq. 9).  beta = 0 (the default) is the exact-match
+ * verification of Eq. 7.  With beta >= 1, a block position keeps its DRAFTED token as the verified token when
+ *   (Eq. 8) fewer than beta other vocabulary entries score strictly higher than the draft, i.e. the draft's
+ *           log-likelihood is at least that of the beta-th ranked token, and
+ *   (Eq. 9) the top-1 score exceeds the draft's score by at most tau (log-likelihoods of one position differ from
+ *           the scores by a common constant, so the gap is taken on the scores),
+ * and the greedy choice otherwise; n_accepted is then taken as before (first position whose verified token
+ * differs from the draft, cut at an accepted [EOS]).  A sentinel draft (negative) never qualifies.  The output is
+ * no longer bound to equal greedy decoding.  Applies to every later ad_verify_block and ad_generate of the
+ * handle (host-side setting, no device work).  tau >= 0.  Errors: AD_ERR_ARG. */
+int ad_set_acceptance(ad_handle* h, int32_t beta, float tau);
+
 /* Waits for the handle's stream; returns and clears a latched device error. */
 int ad_sync(ad_handle* h);
 

@@ -20,7 +20,7 @@ AD_MODE_IAD, AD_MODE_GAD = 0, 1
 
 EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
-    "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync",
+    "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync", "ad_set_acceptance",
     "ad_debug_logits", "ad_debug_encoder_memory", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
     "ad_vocab_argmax_static", "ad_debug_wait_probe",
     "ad_linear",
@@ -86,6 +86,7 @@ def load():
         "ad_draft_block": (C.c_int, [vp, i32, vp, vp, i32]),
         "ad_get_state": (C.c_int, [vp, vp, vp, vp]),
         "ad_sync": (C.c_int, [vp]),
+        "ad_set_acceptance": (C.c_int, [vp, C.c_int32, C.c_float]),
         "ad_debug_logits": (C.c_int, [vp, i32, vp, sz]),
         "ad_debug_encoder_memory": (C.c_int, [vp, i32, vp, sz]),
         "ad_vocab_argmax_scratch_bytes": (sz, [i32, i32]),
@@ -236,6 +237,10 @@ class AggressiveDecoder:
 
     def sync(self):
         self._check(self.lib.ad_sync(self.h), self.h)
+
+    def set_acceptance(self, beta, tau):
+        """beta = 0: exact-match verification; beta >= 1: relaxed top-beta / tau verification."""
+        self._check(self.lib.ad_set_acceptance(self.h, int(beta), float(tau)), self.h)
 
     def debug_logits(self, M, which=0):
         t = self.torch.empty((M, self.shape.vocab), dtype=self.torch.float32, device=self.dev)

@@ -93,6 +93,11 @@ struct ad_handle {
   void *qbuf = nullptr, *ktmp = nullptr, *vtmp = nullptr, *kself = nullptr, *vself = nullptr, *encmem = nullptr;
   float* part_val = nullptr;
   int* part_idx = nullptr;
+  int* part_cnt = nullptr;   // relaxed verification: per tile and token, other tokens scoring above the draft
+  float* draft_val = nullptr;
+  int* draft_id = nullptr;
+  int beta = 0;              // 0: exact-match verification; >= 1: relaxed verification (Section 3.2.3)
+  float tau = 0.f;
   int n_vtiles = 0;
   float* pe = nullptr;
   int max_pos = 0;
@@ -236,6 +241,9 @@ size_t layout(ad_handle* h, void* base) {
   h->n_vtiles = (c.vocab + 127) / 128;
   h->part_val = (float*)bp.take(sizeof(float) * (size_t)h->n_vtiles * Mv);
   h->part_idx = (int*)bp.take(sizeof(int) * (size_t)h->n_vtiles * Mv);
+  h->part_cnt = (int*)bp.take(sizeof(int) * (size_t)h->n_vtiles * Mv);
+  h->draft_val = (float*)bp.take(sizeof(float) * (size_t)Mv);
+  h->draft_id = (int*)bp.take(sizeof(int) * (size_t)Mv);
   h->max_pos = std::max(c.max_src, c.max_tgt + 1);
   h->pe = (float*)bp.take(sizeof(float) * (size_t)h->max_pos * d);
   h->ovr = (int*)bp.take(sizeof(int) * (size_t)B * c.max_tgt);
@@ -601,11 +609,21 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
   PassCfg& pc = h->pass[PK_VERIFY];
   GemmParams p = {};
   p.part_val = h->part_val; p.part_idx = h->part_idx;
+  const int beta = to_drafts ? 0 : h->beta;
+  if (beta >= 1) {   // relaxed verification: the drafts' own scores first, then the projection counts against them
+    const int d = h->cfg.d_model;
+    h->launches++;
+    const dim3 sgrid((pc.M_cap + 7) / 8);
+    if (h->bf16) AD_CUDA(h, launch_k(draft_score_kernel<bf16, bf16>, sgrid, dim3(256), 0, h->stream, h->st, pc.plan, h->dims, (const bf16*)m.emb.ptr, (const bf16*)X.ptr, d, h->draft_val, h->draft_id));
+    else AD_CUDA(h, launch_k(draft_score_kernel<float, float>, sgrid, dim3(256), 0, h->stream, h->st, pc.plan, h->dims, (const float*)m.emb.ptr, (const float*)X.ptr, d, h->draft_val, h->draft_id));
+    p.draft_val = h->draft_val; p.draft_id = h->draft_id; p.part_cnt = h->part_cnt;
+  }
   AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   h->launches++;
   AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
                       pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
-                      auto_commit ? h->cond_handle : 0ull));
+                      auto_commit ? h->cond_handle : 0ull, beta, h->tau, (const float*)h->draft_val, (const int*)h->draft_id,
+                      (const int*)h->part_cnt));
   h->last_vocab_which = to_drafts ? 1 : 0;
   return AD_OK;
 }
@@ -774,6 +792,14 @@ extern "C" int ad_destroy(ad_handle* h) {
   if (h->ev1) cudaEventDestroy(h->ev1);
   if (h->ev2) cudaEventDestroy(h->ev2);
   delete h;
+  return AD_OK;
+}
+
+extern "C" int ad_set_acceptance(ad_handle* h, int32_t beta, float tau) {
+  if (!h) return AD_ERR_ARG;
+  if (beta < 0 || !(tau >= 0.f)) return fail(h, AD_ERR_ARG, "beta must be >= 0 and tau >= 0");
+  h->beta = beta;
+  h->tau = tau;
   return AD_OK;
 }
 
@@ -962,7 +988,8 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
   bool device_loop = false;
   if (opts->use_graph && h->stream != nullptr) {   // the legacy default stream cannot be captured
     char key[160];
-    snprintf(key, sizeof(key), "B%d m%d k%d o%d v%d d%d", B, opts->mode, opts->k, ovr ? 1 : 0, ovr_len, opts->run_drafter);
+    snprintf(key, sizeof(key), "B%d m%d k%d o%d v%d d%d b%d t%a", B, opts->mode, opts->k, ovr ? 1 : 0, ovr_len, opts->run_drafter,
+             h->beta, (double)h->tau);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
       const int before = h->launches;

@@ -70,6 +70,11 @@ struct GemmParams {
   // EPI_ARGMAX
   float* part_val;       // [M_cap, n_tiles]: per token, the best value of every 128-feature tile
   int* part_idx;         // [M_cap, n_tiles]
+  // EPI_ARGMAX with the relaxed verification (null: off): per token, the drafted token and its score; the kernel
+  // adds, per feature tile, how many OTHER features score strictly higher than the draft
+  const float* draft_val;  // [M_cap]
+  const int* draft_id;     // [M_cap] (negative: no draft at this position)
+  int* part_cnt;           // [M_cap, n_tiles]
   int* status;           // device status word (latches AD_ERR_TIMEOUT), may be null
 };
 

@@ -22,6 +22,7 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
   __shared__ float xs[TOK][KT];
   __shared__ float red_val[4][TOK];
   __shared__ int red_idx[4][TOK];
+  __shared__ int red_cnt[4][TOK];
 
   pdl_launch();
   pdl_wait();
@@ -67,6 +68,12 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
     for (int j = 0; j < TOK; ++j) {
       float v = (n < p.N) ? acc[j] : -INFINITY;
       int i = n;
+      if (p.draft_val) {   // relaxed verification: features other than the draft that score strictly higher
+        const bool on = t0 + j < M;
+        const bool above = on && n < p.N && n != p.draft_id[t0 + j] && acc[j] > p.draft_val[t0 + j];
+        const unsigned int bal = __ballot_sync(0xffffffffu, above);
+        if (lane == 0) red_cnt[warp][j] = __popc(bal);
+      }
       tc::warp_argmax(v, i);
       if (lane == 0) { red_val[warp][j] = v; red_idx[warp][j] = i; }
     }
@@ -82,6 +89,9 @@ gemm_f32_kernel(const float* __restrict__ w, const float* __restrict__ x, const 
       }
       p.part_val[(size_t)(t0 + tid) * gridDim.x + blockIdx.x] = v;
       p.part_idx[(size_t)(t0 + tid) * gridDim.x + blockIdx.x] = i;
+      if (p.draft_val)
+        p.part_cnt[(size_t)(t0 + tid) * gridDim.x + blockIdx.x] =
+            red_cnt[0][tid] + red_cnt[1][tid] + red_cnt[2][tid] + red_cnt[3][tid];
     }
   } else {
     __shared__ int slot_s[TOK];

@@ -264,6 +264,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ int slot_s[256];
+  __shared__ float dval_s[256];   // relaxed verification: score and id of every token's draft
+  __shared__ int did_s[256];
 
   trace_mark(TR_GEMM + EPI, 0);
   const int ntile = p.ntile;
@@ -339,6 +341,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   if (valid) {
     if (EPI == EPI_SCATTER) {
       for (int j = threadIdx.x; j < ntile; j += THREADS) slot_s[j] = (t0 + j < M) ? p.slot[t0 + j] : 0;
+    }
+    if (EPI == EPI_ARGMAX && p.draft_val) {
+      for (int j = threadIdx.x; j < ntile; j += THREADS) {
+        dval_s[j] = (t0 + j < M) ? p.draft_val[t0 + j] : 0.f;
+        did_s[j] = (t0 + j < M) ? p.draft_id[t0 + j] : -1;
+      }
     }
     if (lane == 0 && warp != 1 && warp < 4) {
       // ---- TMA producers: everything that was not issued above ----
@@ -427,6 +435,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       // meet in shared memory and one thread per token combines them in ascending feature order.
       float* red_val = stage;                                   // [4][ntile]
       int* red_idx = reinterpret_cast<int*>(stage + 4 * 256);   // [4][ntile]
+      int* red_cnt = reinterpret_cast<int*>(stage + 8 * 256);   // [4][ntile] features scoring above the draft
+      const bool relaxed = p.draft_val != nullptr;
       if (ready) {
         for (int c = grp * 16; c < ntile && c < ntok_all; c += 32) {
           float acc[16];
@@ -434,6 +444,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           // columns past the last valid token hold whatever the padded activation rows produced: never stored
 #pragma unroll
           for (int j = 0; j < 16; ++j) acc[j] = n < p.N ? acc[j] + bias_n : -INFINITY;
+          int my_cnt = 0;
+          if (relaxed) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int tt = c + j;
+              const bool above = tt < ntok_all && n < p.N && n != did_s[tt] && acc[j] > dval_s[tt];
+              const unsigned int bal = __ballot_sync(0xffffffffu, above);
+              if ((lane >> 1) == j) my_cnt = __popc(bal);
+            }
+          }
           float my_v;
           int my_i;
           warp_argmax_items16(acc, lane, my_v, my_i);
@@ -441,6 +461,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           if (!(lane & 1) && t < ntok_all) {
             red_val[quad * ntile + t] = my_v;
             red_idx[quad * ntile + t] = n0 + quad * 32 + my_i;
+            if (relaxed) red_cnt[quad * ntile + t] = my_cnt;
           }
         }
       }
@@ -456,6 +477,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
         p.part_val[(size_t)(t0 + t) * gridDim.x + blockIdx.x] = v;
         p.part_idx[(size_t)(t0 + t) * gridDim.x + blockIdx.x] = idx;
+        if (relaxed)
+          p.part_cnt[(size_t)(t0 + t) * gridDim.x + blockIdx.x] =
+              red_cnt[t] + red_cnt[ntile + t] + red_cnt[2 * ntile + t] + red_cnt[3 * ntile + t];
       }
     }
     // Other epilogues: the tile is transposed through shared memory into rows of 128 features per token, in

@@ -513,11 +513,39 @@ __device__ __forceinline__ void finish_iteration(const DevState& st, const Dims&
 }
 
 // ---------------------------------------------------------------------------------------------
+// Relaxed verification (Section 3.2.3): score of every block position's drafted token,
+// draft_val[m] = x[m, :] . emb[draft, :], and its id (negative: sentinel, never kept).  The projection kernel
+// then counts, per position, the other tokens that score strictly higher (Eq. 8), and the accept kernel applies
+// Eq. 8 and Eq. 9.  One warp per packed token; grid = ceil(M_cap / 8), block = 256.
+// ---------------------------------------------------------------------------------------------
+template <typename WT, typename ActT>
+__global__ void __launch_bounds__(256)
+draft_score_kernel(DevState st, PassPlan blk, Dims dm, const WT* __restrict__ emb, const ActT* __restrict__ x, int d,
+                   float* __restrict__ draft_val, int* __restrict__ draft_id) {
+  pdl_launch();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * 8 + warp;
+  if (m >= *blk.M) return;
+  const int b = blk.tok_row[m];
+  const int id = st.drafts[(size_t)b * dm.kmax + (m - blk.seg_off[b])];
+  float acc = 0.f;
+  if (id >= 0)
+    for (int i = lane; i < d; i += 32) acc = fmaf(to_f32(x[(size_t)m * d + i]), to_f32(emb[(size_t)id * d + i]), acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) { draft_val[m] = acc; draft_id[m] = id; }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Final arg-max over the per-tile partials of the fused projection, then the draft compare:
 //   c = first block position whose greedy choice differs from the draft (Section 3.1.1; definition of c
 //   in Section 3.2), n = c + 1 (the bifurcation token is kept), n = k when nothing differs, cut at the
 //   first accepted [EOS].  One CTA per row, one warp per block position for the reduction; warp 0 takes the
 //   decision with ballots.
+// beta >= 1: relaxed verification of Section 3.2.3 -- a position keeps its drafted token when fewer than beta other
+//   tokens score strictly higher (Eq. 8: the draft is within the top beta) and the best score exceeds the draft's
+//   by at most tau (Eq. 9; differences of log-likelihoods are differences of scores); otherwise the greedy choice.
 // to_drafts != 0: drafter mode, the choices are written as the row's drafts and nothing is compared.
 // auto_commit != 0: the row's n_accepted is committed right away (decode loop); the last CTA to finish
 //   updates the loop counter and the all-finished word (done_ctr: rows done in the low half, active rows in
@@ -527,7 +555,9 @@ __device__ __forceinline__ void finish_iteration(const DevState& st, const Dims&
 __global__ void __launch_bounds__(1024)
 argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
                      const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts, int auto_commit,
-                     unsigned int* done_ctr, unsigned long long cond) {
+                     unsigned int* done_ctr, unsigned long long cond, int beta, float tau,
+                     const float* __restrict__ draft_val, const int* __restrict__ draft_id,
+                     const int* __restrict__ part_cnt) {
   trace_mark(TR_ACCEPT, 0);
   pdl_launch();
   pdl_wait();
@@ -542,18 +572,29 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
       const int m = off + i;
       float v = -INFINITY;
       int idx = 0x7fffffff;
+      int higher = 0;
+      const bool relaxed = beta >= 1 && !to_drafts;
       for (int t = lane; t < n_tiles; t += 32) {
         const float ov = part_val[(size_t)m * n_tiles + t];
         const int oi = part_idx[(size_t)m * n_tiles + t];
         if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+        if (relaxed) higher += part_cnt[(size_t)m * n_tiles + t];
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, v, o);
         const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
         if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+        higher += __shfl_xor_sync(0xffffffffu, higher, o);
       }
-      if (lane == 0) pred[i] = idx;
+      if (lane == 0) {
+        int choice = idx;
+        if (relaxed) {
+          const int did = draft_id[m];
+          if (did >= 0 && higher <= beta - 1 && v - draft_val[m] <= tau) choice = did;
+        }
+        pred[i] = choice;
+      }
     }
   }
   if (to_drafts) return;

@@ -1,0 +1,193 @@
+"""Parity of the relaxed verification (Section 3.2.3: top-beta / tau requirement) with the CPU checker, through
+the C ABI: block level on an FP32 and a BF16 model, whole loop on the FP32 model, and the setter's edge cases.
+
+The decision "keep the draft" depends on score comparisons, so ids are compared exactly only where the checker
+reports that no comparison is closer than the margin (0.1 for BF16 scores, whose bar is 5e-2 max-abs; 1e-2 for
+FP32 scores, whose bar is 1e-3); elsewhere n_accepted must at least be the accept rule applied to the library's own
+verified tokens.
+"""
+import numpy as np
+import pytest
+
+from oracle import ad_oracle as O
+from paper_2205_10350_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+OPS = O.Ops("f32")
+SETTINGS = [(1, 0.0), (3, 0.05), (5, 0.3), (5, 3.0), (2000, 1e30)]
+
+
+def make(shape, max_src, max_tgt, kmax, batch=1):
+    w = synth.make_weights(shape, 0)
+    dec = binding.AggressiveDecoder(shape, w, None, max_batch=batch, max_src=max_src, max_tgt=max_tgt, kmax=kmax)
+    om = O.Model(shape, w, max_pos=max(max_src, max_tgt + 1))
+    return dec, om
+
+
+def mixed_drafts(st, g, k, r, vocab):
+    """Greedy tokens, runner-ups of the checker's own scores, noise and one sentinel."""
+    st.reset()
+    lg = st.verify_block(0, g[:k], want_logits=True)["logits"]
+    d = np.asarray(g[:k], np.int32).copy()
+    for i in range(k):
+        u = r.random()
+        if u < 0.4:
+            d[i] = np.argsort(-lg[i], kind="stable")[int(r.integers(1, 6))]
+        elif u < 0.5:
+            d[i] = int(r.integers(4, vocab))
+    d[d == 2] = 5
+    return d
+
+
+def check_block(dec, st, d, beta, tau, margin, tol):
+    k = len(d)
+    st.reset()
+    res = st.verify_block_pp(0, d, beta, tau, want_logits=True)
+    drafts = np.full((1, dec.kmax), -1, np.int32)
+    drafts[0, :k] = d
+    dec.set_acceptance(beta, tau)
+    ids, n = dec.verify_block(drafts, [k])
+    lg = dec.debug_logits(k)
+    assert np.abs(lg - res["logits"]).max() <= tol
+    clear = np.zeros(k, bool)
+    for i in range(k):
+        clear[i] = res["dmargin"][i] > margin and (res["met"][i] or res["margin"][i] > margin)
+        if clear[i]:
+            assert ids[0, i] == res["pred"][i], (beta, tau, i, ids[0, i], res["pred"][i], res["dmargin"][i])
+        else:                                  # either the draft or one of the checker's top two
+            top2 = np.argsort(-res["logits"][i], kind="stable")[:2]
+            assert ids[0, i] == d[i] or ids[0, i] in top2
+    n_self, _ = OPS.accept(ids[0, :k], d, eos=2)
+    assert n[0] == n_self
+    if clear[: res["n"]].all():
+        assert n[0] == res["n"]
+    return int(clear.sum()), int(res["met"].sum())
+
+
+def test_fp32_block_parity():
+    dec, om = make(synth.TINY, 16, 24, 17)
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    st = om.state(src[0, : lens[0]])
+    g, _ = st.greedy(24)
+    dec.encode(src, lens)
+    r = np.random.default_rng(21)
+    seen_clear = seen_met = 0
+    for beta, tau in SETTINGS:
+        for _ in range(3):
+            d = mixed_drafts(st, g, 12, r, synth.TINY.vocab)
+            d[-1] = -1
+            c, m = check_block(dec, st, d, beta, tau, 1e-2, 1e-3)
+            seen_clear += c
+            seen_met += m
+    assert seen_clear > 100 and seen_met > 40
+    # back to the exact-match rule on the same handle
+    dec.set_acceptance(0, 0.0)
+    d = mixed_drafts(st, g, 12, r, synth.TINY.vocab)
+    st.reset()
+    ref = st.verify_block(0, d)
+    drafts = np.full((1, dec.kmax), -1, np.int32)
+    drafts[0, :12] = d
+    ids, n = dec.verify_block(drafts, [12])
+    assert np.array_equal(ids[0, :12], ref["pred"]) and n[0] == ref["n"]
+    dec.close()
+
+
+def test_bf16_block_parity_several_tiles():
+    """MINI BF16 model, vocabulary 2048 = 16 projection tiles, blocks of 20 tokens (ragged against the 32-token tile)."""
+    shape = synth.MINI_BF16
+    dec, om = make(shape, 12, 24, 20)
+    src = np.array([[5, 9, 700, 33, 1200, 8, 64, 65, 77, 78, 79, 80]], np.int32)
+    lens = np.array([12], np.int32)
+    st = om.state(src[0])
+    g, _ = st.greedy(24)
+    dec.encode(src, lens)
+    r = np.random.default_rng(22)
+    seen_clear = seen_met = 0
+    for beta, tau in SETTINGS:
+        for _ in range(2):
+            d = mixed_drafts(st, g, min(20, len(g)), r, shape.vocab)
+            c, m = check_block(dec, st, d, beta, tau, 0.1, 5e-2)
+            seen_clear += c
+            seen_met += m
+    assert seen_clear > 40 and seen_met > 20
+    dec.close()
+
+
+@pytest.mark.parametrize("beta,tau", [(3, 0.05), (5, 0.3), (1000, 1e30)])
+def test_fp32_loop_parity(beta, tau):
+    dec, om = make(synth.TINY, 16, 24, 17)
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    st = om.state(src[0, : lens[0]])
+    g, _ = st.greedy(24)
+    stream = synth.corrupt_stream(g[None, :], [len(g)], 0.6, synth.TINY.vocab, 3)[0]
+    ref, tr = st.gad_pp(None, 6, 24, beta, tau, override=stream)
+    dec.set_acceptance(beta, tau)
+    ov = np.full((1, 24), -1, np.int32)
+    ov[0, : len(stream)] = stream
+    for graph in (False, True):
+        outs, stats = dec.generate(src, lens, mode="GAD", k=6, max_len=[24], draft_override=ov, use_graph=graph)
+        out = outs[0]
+        n = min(len(out), len(ref))
+        diff = np.nonzero(out[:n] != ref[:n])[0]
+        if len(diff) == 0:
+            assert len(out) == len(ref) and stats["iterations"] == tr["iterations"]
+        else:                                  # the first difference must sit at a knife-edge decision
+            p = int(diff[0])
+            lg = om.decode_full(om.encode_memory(st.src), np.concatenate([[0], ref[:p]]).astype(np.int32))
+            _, _, tm, dm = OPS.relaxed_choice(lg[p], int(stream[p]) if p < len(stream) else -1, beta, tau)
+            assert min(tm, dm) <= 1e-2, (p, tm, dm)
+    # the exact-match rule after the relaxed one: greedy again
+    dec.set_acceptance(0, 0.0)
+    outs, _ = dec.generate(src, lens, mode="GAD", k=6, max_len=[24], draft_override=ov)
+    assert np.array_equal(outs[0], g)
+    dec.close()
+
+
+def test_setter_rejects_bad_values():
+    dec, _ = make(synth.TINY, 16, 24, 17)
+    for beta, tau in ((-1, 0.0), (1, -0.5), (1, float("nan"))):
+        with pytest.raises(binding.AdError):
+            dec.set_acceptance(beta, tau)
+    dec.set_acceptance(3, 0.25)
+    dec.close()
+
+
+def test_bf16_base_two_ragged_rows():
+    """Transformer-base (vocabulary 32000 = 250 projection tiles), two rows with blocks of 12 and 7 tokens packed into
+    one pass: the relaxed rule is applied per row with the row's own drafts."""
+    shape = synth.BASE
+    dec, om = make(shape, 16, 16, 12, batch=2)
+    r = np.random.default_rng(23)
+    src = r.integers(4, shape.vocab, size=(2, 16)).astype(np.int32)
+    lens = np.array([16, 11], np.int32)
+    sts = [om.state(src[b, : lens[b]]) for b in range(2)]
+    ks = [12, 7]
+    dec.encode(src, lens)
+    beta, tau = 4, 0.25
+    dec.set_acceptance(beta, tau)
+    drafts = np.full((2, dec.kmax), -1, np.int32)
+    refs = []
+    for b in range(2):
+        g, _ = sts[b].greedy(ks[b])
+        d = mixed_drafts(sts[b], g, ks[b], r, shape.vocab)
+        drafts[b, : ks[b]] = d
+        sts[b].reset()
+        refs.append(sts[b].verify_block_pp(0, d, beta, tau, want_logits=True))
+    ids, n = dec.verify_block(drafts, ks)
+    lg = dec.debug_logits(sum(ks))
+    off, clear_total = 0, 0
+    for b in range(2):
+        res, k, d = refs[b], ks[b], drafts[b, : ks[b]]
+        assert np.abs(lg[off: off + k] - res["logits"]).max() <= 5e-2
+        clear = (res["dmargin"] > 0.1) & (res["met"] | (res["margin"] > 0.1))
+        for i in range(k):
+            if clear[i]:
+                assert ids[b, i] == res["pred"][i], (b, i)
+        n_self, _ = OPS.accept(ids[b, :k], d, eos=2)
+        assert n[b] == n_self
+        if clear[: res["n"]].all():
+            assert n[b] == res["n"]
+        clear_total += int(clear.sum())
+        off += k
+    assert clear_total >= 6
+    dec.close()
