@@ -18,7 +18,8 @@ import torch
 
 from . import binding, synth
 
-MODELS = {"tiny": synth.TINY, "base": synth.BASE, "big": synth.BIG, "mini": synth.MINI_BF16}
+MODELS = {"tiny": synth.TINY, "base": synth.BASE, "big": synth.BIG, "mini": synth.MINI_BF16,
+          "deep12_2": synth.DEEP_ENC, "bart_base": synth.BART_BASE_SIZED}
 
 
 def _events(stream, fn, reps, flush=None):

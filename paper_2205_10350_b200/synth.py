@@ -47,6 +47,10 @@ class ModelShape:
 TINY = ModelShape("tiny", 128, 4, 512, 1000, 2, 2, "fp32")
 BASE = ModelShape("base", 512, 8, 2048, 32000, 6, 6, "bf16")
 BIG = ModelShape("big", 1024, 16, 4096, 32000, 6, 6, "bf16")
+# Further shapes the paper reports on (Section 4.1.2: a 12-layer encoder with a 2-layer decoder; Section 4.2.4:
+# models of the size of BART-base); same kernels, other layer counts and widths.
+DEEP_ENC = ModelShape("deep_encoder_12_2", 512, 8, 2048, 32000, 12, 2, "bf16")
+BART_BASE_SIZED = ModelShape("bart_base_sized", 768, 12, 3072, 50265, 6, 6, "bf16")
 # A small bf16 shape for fast tests of the tensor-core path (not one of the five workloads).
 MINI_BF16 = ModelShape("mini_bf16", 256, 4, 512, 2048, 2, 2, "bf16")
 

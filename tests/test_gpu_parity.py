@@ -257,3 +257,44 @@ def test_long_source_short_blocks(base_weights):
             streams[b, 6] = 13
         tot = P.lockstep(dec, om, src, lens, list(streams), kmax, [40, 40], TOL_BF16, max_steps=2)
         assert tot["steps"] == 2
+
+
+# ------------------------------------------------------------------------------------------ other shapes
+def test_deep_encoder_shallow_decoder_shape():
+    """A 6-layer encoder over a 1-layer decoder (the layer split of the paper's 12+2 model, Section 4.1.2, at a width
+    the checker finishes in seconds): input-guided lock-step run and free run."""
+    shape = synth.ModelShape("deep_enc_mini", 256, 4, 512, 2048, 6, 1, "bf16")
+    dec, om, _ = make(shape, 2, 18, 20, 19)
+    wl = synth.Workload(10, shape, "IAD", 2, 1, 10, 18, 0, 19, 0.85, False)
+    src, lens = synth.make_sources(wl)
+    max_len = np.minimum(lens, 20)
+    greedy = [om.state(src[b, : lens[b]]).greedy(int(max_len[b])) for b in range(2)]
+    g = np.full((2, 20), synth.PAD, np.int32)
+    for b in range(2):
+        g[b, : len(greedy[b][0])] = greedy[b][0]
+    streams = synth.corrupt_stream(g, max_len, 0.85, shape.vocab, 10)
+    tot = P.lockstep(dec, om, src, lens, list(streams), 19, max_len, TOL_BF16)
+    assert tot["tokens"] == int(sum(len(x[0]) for x in greedy))
+    outs, _ = dec.generate(src, lens, mode="IAD", k=19, max_len=max_len)       # Algorithm 1 on the real sources
+    for b in range(2):
+        P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"row {b}")
+    dec.close()
+
+
+def test_bart_base_sized_shape_two_steps():
+    """d_model 768, 12 heads, FFN 3072, vocabulary 50265 (393 projection tiles, the last one ragged), the size of the
+    models of Section 4.2.4: encoder memory and two lock-step verification steps of a 10-token block."""
+    shape = synth.BART_BASE_SIZED
+    dec, om, _ = make(shape, 1, 24, 24, 10)
+    r = np.random.default_rng(31)
+    src = r.integers(4, shape.vocab, size=(1, 24)).astype(np.int32)
+    lens = np.array([24], np.int32)
+    st = om.state(src[0])
+    g, _ = st.greedy(20)
+    stream = synth.corrupt_stream(g[None, :], [len(g)], 0.8, shape.vocab, 31)[0]
+    dec.encode(src, lens)
+    mem = dec.debug_encoder_memory(0, 24)
+    assert np.abs(mem - st.memory()).max() < 5e-2
+    tot = P.lockstep(dec, om, src, lens, [stream], 10, [20], TOL_BF16, max_steps=2)
+    assert tot["steps"] == 2 and tot["worst_logit_err"] < TOL_BF16
+    dec.close()
