@@ -229,7 +229,10 @@ int ad_debug_wait_probe(int32_t* status, int32_t poll_limit, int32_t* polls_done
 /* Output projection fused with the row arg-max (Eq. 3 / Eq. 7 "top-1"): for each of M rows of x [M, d]
  * (dtype as given) against emb [vocab, d], argmax[m] = lowest id with the largest score; the scores are
  * never written.  scratch: device memory for per-tile partial maxima, ad_vocab_argmax_scratch_bytes().
- * status: optional device int that latches AD_ERR_TIMEOUT.  BF16 needs d % 64 == 0 and M <= 256. */
+ * status: optional device int that latches AD_ERR_TIMEOUT.  BF16 needs d % 64 == 0 and M <= 256.
+ * argmax == NULL runs the projection kernel alone and leaves its per-tile (maximum, id) partials in scratch
+ * (values [M, tiles] FP32 first, ids [M, tiles] int32 from the next 256-byte boundary, tiles = ceil(vocab / 128)):
+ * the launch a micro-benchmark times when it wants the projection without the final reduction. */
 size_t ad_vocab_argmax_scratch_bytes(int32_t vocab, int32_t M);
 int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d, int32_t vocab,
                     int32_t* argmax, void* scratch, size_t scratch_bytes, int32_t* status, void* stream);

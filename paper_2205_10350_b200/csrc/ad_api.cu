@@ -1189,7 +1189,7 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part_val, const int
 
 extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, int32_t M, int32_t d, int32_t vocab,
                                int32_t* argmax, void* scratch, size_t scratch_bytes, int32_t* status, void* stream) {
-  if (!x || !emb || !argmax || !scratch || M < 1 || d < 1 || vocab < 1) return AD_ERR_ARG;
+  if (!x || !emb || !scratch || M < 1 || d < 1 || vocab < 1) return AD_ERR_ARG;
   if (scratch_bytes < ad_vocab_argmax_scratch_bytes(vocab, M)) return AD_ERR_CAPACITY;
   if (reinterpret_cast<uintptr_t>(scratch) % 256) return AD_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1212,6 +1212,7 @@ extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, in
     return AD_ERR_ARG;
   }
   if (e != cudaSuccess) return AD_ERR_CUDA;
+  if (!argmax) return AD_OK;   // projection kernel alone: partials stay in scratch
   e = launch_k(argmax_rows_kernel, dim3(M), dim3(32), 0, st, (const float*)pv, (const int*)pi, tiles, M, argmax);
   return e == cudaSuccess ? AD_OK : AD_ERR_CUDA;
 }
