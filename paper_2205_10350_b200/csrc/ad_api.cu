@@ -89,6 +89,7 @@ struct ad_handle {
   DevState st;
   // activations
   float *y = nullptr, *pre = nullptr;
+  float* pre2 = nullptr;     // per-head partial sums of an output projection fused into the attention kernel
   ActBuf yb, abuf, hbuf, xg;
   void *qbuf = nullptr, *ktmp = nullptr, *vtmp = nullptr, *kself = nullptr, *vself = nullptr, *encmem = nullptr;
   float* part_val = nullptr;
@@ -220,6 +221,7 @@ size_t layout(ad_handle* h, void* base) {
   size_t pre_elems = 0;
   for (int k = 0; k < PK_COUNT; ++k) pre_elems = std::max(pre_elems, (size_t)h->pass[k].max_split * h->pass[k].M_cap * d);
   h->pre = (float*)bp.take(sizeof(float) * pre_elems);
+  if (h->bf16 && c.n_heads <= 16) h->pre2 = (float*)bp.take(sizeof(float) * (size_t)c.n_heads * M_all * d);
   h->yb.ptr = bp.take(e * (size_t)M_all * d); h->yb.cols = d;
   h->abuf.ptr = bp.take(e * (size_t)M_all * d); h->abuf.cols = d;
   h->hbuf.ptr = bp.take(e * (size_t)M_all * F); h->hbuf.cols = F;
@@ -324,6 +326,7 @@ int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
 bool g_use_pdl = true;       // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
 bool g_use_graph_encode = true;   // AD_NO_ENCODE_GRAPH=1: launch the encoder kernels directly
 bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
+bool g_fuse_attn_proj = true;   // AD_NO_ATTN_PROJ=1: attention and its output projection always as separate kernels
 
 // Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
 // themselves wait with griddepcontrol.wait before touching anything a predecessor writes).
@@ -410,21 +413,21 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   return AD_OK;
 }
 
-template <typename T, int D, int Q>
+template <typename T, int D, int Q, bool FUSE = false>
 cudaError_t launch_attention(dim3 grid, dim3 block, cudaStream_t st, const AttnParams& p) {
   constexpr size_t smem = att_smem_bytes<D, Q>();
   static bool attr_set = false;
   if (!attr_set && smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   attr_set = true;
-  return launch_k(attention_kernel<T, D, Q>, grid, block, smem, st, p);
+  return launch_k(attention_kernel<T, D, Q, FUSE>, grid, block, smem, st, p);
 }
 
 int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, const void* v, void* out,
               const int* key_base, const int* nkeys_tok, const int* nkeys_row, int max_keys,
-              const float* q_bias = nullptr, int q_nsplit = 0) {
+              const float* q_bias = nullptr, int q_nsplit = 0, const Mat* wo = nullptr, bool* fused = nullptr) {
   const ad_model_cfg& c = h->cfg;
   AttnParams p;
   p.q = q; p.k = k; p.v = v; p.out = out;
@@ -460,7 +463,14 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   h->launches++;
   cudaError_t e;
 #define AD_ATT(T, D, Q) launch_attention<T, D, Q>(grid, block, h->stream, p)
-  if (h->bf16) {
+  // few queries, 64-wide heads: the output projection rides along (one partial sum per head for the LayerNorm kernel)
+  const bool fuse = g_fuse_attn_proj && wo && fused && h->pre2 && h->bf16 && dh == 64 && !many && c.n_heads <= pc.max_split &&
+                    c.n_heads <= 16 && c.d_model % 128 == 0;
+  if (fused) *fused = fuse;
+  if (fuse) {
+    p.wo = (const bf16*)wo->ptr; p.o_part = h->pre2; p.o_stride = (size_t)pc.M_cap * c.d_model;
+    e = launch_attention<bf16, 64, 1, true>(grid, block, h->stream, p);
+  } else if (h->bf16) {
     if (dh == 64) e = many ? AD_ATT(bf16, 64, 8) : AD_ATT(bf16, 64, 1);
     else e = many ? AD_ATT(bf16, 32, 8) : AD_ATT(bf16, 32, 1);
   } else {
@@ -473,7 +483,9 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
 }
 
 // y = LN(sum of the nsplit partial projections in `pre` + bias + y)
-int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, const float* g, const float* b) {
+int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, const float* g, const float* b,
+              const float* partials = nullptr) {
+  const float* pre_src = partials ? partials : h->pre;
   const int d = h->cfg.d_model;
   dim3 grid(pc.M_cap);
   const size_t stride = (size_t)pc.M_cap * d;
@@ -481,13 +493,13 @@ int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, co
   cudaError_t e;
   if (pc.M_cap >= 512 && d % 128 == 0 && d <= 1024) {   // many tokens: a warp per token
     dim3 rgrid((pc.M_cap + 7) / 8);
-    if (h->bf16) e = launch_k(layernorm_rows_kernel<bf16>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+    if (h->bf16) e = launch_k(layernorm_rows_kernel<bf16>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                               (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
-    else e = launch_k(layernorm_rows_kernel<float>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+    else e = launch_k(layernorm_rows_kernel<float>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                       (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
-  } else if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+  } else if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                             (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
-  else e = launch_k(layernorm_kernel<float>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, (const float*)h->pre, nsplit, stride, bias,
+  else e = launch_k(layernorm_kernel<float>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                     (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("layernorm launch: ") + cudaGetErrorString(e));
   return AD_OK;
@@ -525,8 +537,10 @@ int self_attention_sublayer(ad_handle* h, int pk, const Mat& wqkv, const float* 
   p.bias = bqkv; p.dst[0] = h->qbuf; p.dst[1] = kbuf; p.dst[2] = vbuf; p.seg_width = h->cfg.d_model; p.n_direct = 1;
   p.slot = pc.plan.kv_slot;
   AD_TRY(gemm(h, EPI_SCATTER, wqkv, h->yb, pk, pc.plan.M, pc.M_cap, p));
+  bool fused = false;
   AD_TRY(attention(h, pc, h->qbuf, kbuf, vbuf, h->abuf.ptr, pc.plan.key_base, pc.plan.att_n, pc.plan.row_nk,
-                   pk == PK_VERIFY ? h->dims.max_tgt : pc.seg_max));
+                   pk == PK_VERIFY ? h->dims.max_tgt : pc.seg_max, nullptr, 0, &wo, &fused));
+  if (fused) return layernorm(h, pc, h->cfg.n_heads, bo, lng, lnb, h->pre2);
   int ns = 1;
   AD_TRY(gemm_to_ln(h, wo, h->abuf, pk, &ns));
   return layernorm(h, pc, ns, bo, lng, lnb);
@@ -559,22 +573,27 @@ int decoder_pass(ad_handle* h, int pk, Model& m) {
     // Query projection of the cross-attention.  With few tokens a full-K walk per CTA is the slow part of the
     // projection, so it is split along K and the attention kernel adds the partial sums (and the bias) as it
     // loads its queries.
+    bool fused_x = false;
     int qs = h->bf16 && pc.M_cap <= 256 ? pc.ksplit_for(L.cq.N, L.cq.K, pc.tile_for(L.cq.N, num_sms())) : 1;
     if (qs > 1 && qs <= ATT_MAX_QSPLIT) {
       int ns_q = 1;
       AD_TRY(gemm_to_ln(h, L.cq, h->yb, pk, &ns_q));
       AD_TRY(attention(h, pc, nullptr, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
-                       h->st.cross_base, nullptr, h->st.srclen, c.max_src, L.cbq, ns_q));
+                       h->st.cross_base, nullptr, h->st.srclen, c.max_src, L.cbq, ns_q, &L.co, &fused_x));
     } else {
       GemmParams q = {};
       q.bias = L.cbq; q.out_act = h->qbuf;
       AD_TRY(gemm(h, EPI_ACT, L.cq, h->yb, pk, pc.plan.M, pc.M_cap, q));
       AD_TRY(attention(h, pc, h->qbuf, (char*)m.kenc + l * cross_layer, (char*)m.venc + l * cross_layer, h->abuf.ptr,
-                       h->st.cross_base, nullptr, h->st.srclen, c.max_src));
+                       h->st.cross_base, nullptr, h->st.srclen, c.max_src, nullptr, 0, &L.co, &fused_x));
     }
-    int ns = 1;
-    AD_TRY(gemm_to_ln(h, L.co, h->abuf, pk, &ns));
-    AD_TRY(layernorm(h, pc, ns, L.cbo, L.ln2g, L.ln2b));
+    if (fused_x) {
+      AD_TRY(layernorm(h, pc, c.n_heads, L.cbo, L.ln2g, L.ln2b, h->pre2));
+    } else {
+      int ns = 1;
+      AD_TRY(gemm_to_ln(h, L.co, h->abuf, pk, &ns));
+      AD_TRY(layernorm(h, pc, ns, L.cbo, L.ln2g, L.ln2b));
+    }
     AD_TRY(ffn_sublayer(h, pk, L.w1, L.b1, L.w2, L.b2, L.ln3g, L.ln3b));
   }
   return AD_OK;
@@ -736,6 +755,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   { const char* e = getenv("AD_NO_PDL"); g_use_pdl = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_DEVLOOP"); g_use_devloop = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ENCODE_GRAPH"); g_use_graph_encode = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_NO_ATTN_PROJ"); g_fuse_attn_proj = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();

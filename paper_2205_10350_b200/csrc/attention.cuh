@@ -32,7 +32,23 @@ struct AttnParams {
   int d;
   int qchunks;           // query chunks per row = ceil(longest possible segment / queries per CTA)
   float scale;           // 1 / sqrt(head dim)
+  // Fused output projection (FUSE kernels only): instead of storing the attention output, the CTA of head h multiplies
+  // its queries' outputs (rounded to BF16, as a stored output would be) with columns [64 h, 64 h + 64) of wo [d, d]
+  // and writes o_part[h][m, :] = the head's FP32 share of the projection; the residual + LayerNorm kernel adds the
+  // heads up like split-K partials.
+  const bf16* wo;
+  float* o_part;         // [heads][M_cap, d]
+  size_t o_stride;       // M_cap * d
 };
+
+// D (16 x 8, FP32) += A (16 x 16, BF16, row-major) * B (16 x 8, BF16, column-major), warp-level.
+__device__ __forceinline__ void att_mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 
 // Eight consecutive elements (16-byte aligned for bf16, 32-byte for float) as floats.
 __device__ __forceinline__ void load8(const bf16* p, float* out) {
@@ -66,7 +82,11 @@ constexpr size_t att_smem_bytes() {
 // there are few queries; QPW = 8 amortises the K/V staging when there are thousands.
 // Global-memory round trips on the critical path: (1) the row's segment / key-range descriptors,
 // (2) the queries, their key counts and the first K/V tile together, then compute and store.
-template <typename ActT, int DH, int QPW>
+// FUSE (BF16, 64-wide heads, one query per warp): the output projection of the 8 queries is done here as well (see
+// AttnParams::wo).  Warp w owns output features [w d / 8, (w + 1) d / 8); its weight fragments -- 16 rows x 64 columns
+// per group of rows, read with 16-byte loads whose eight elements are consecutive in K (the contraction index is
+// permuted identically for both MMA operands) -- are requested before the dependency wait, since weights never change.
+template <typename ActT, int DH, int QPW, bool FUSE = false>
 __global__ void __launch_bounds__(256)
 attention_kernel(const AttnParams p) {
   constexpr int R = DH / 32;                 // output dims per lane
@@ -80,6 +100,23 @@ attention_kernel(const AttnParams p) {
 
   trace_mark(TR_ATTN, 0);
   pdl_launch();
+  // fused projection: first four row groups of this warp's weight fragments ([group][K chunk][row g / g + 8])
+  uint4 wf[4][2][2];
+  __shared__ __align__(16) bf16 a_s[ATT_WARPS][96];       // the queries' outputs; row stride 192 B: conflict-free 16-byte loads
+  if (FUSE) {
+    const int lane_ = threadIdx.x & 31, g_ = lane_ >> 2, t_ = lane_ & 3;
+    const int nrgw = p.d >> 7;                              // row groups of 16 per warp
+    const bf16* wbase = p.wo + (size_t)((threadIdx.x >> 5) * nrgw * 16 + g_) * p.d + blockIdx.y * DH + 8 * t_;
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        if (r < nrgw) {
+          wf[r][c][0] = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(r * 16) * p.d + c * 32));
+          wf[r][c][1] = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(r * 16 + 8) * p.d + c * 32));
+        }
+      }
+  }
   pdl_wait();
   trace_mark(TR_ATTN, 1);
   const int b = blockIdx.x / p.qchunks;
@@ -212,15 +249,69 @@ attention_kernel(const AttnParams p) {
     __syncwarp();
   }
 
-  ActT* out = reinterpret_cast<ActT*>(p.out);
+  if (FUSE) {
+    // this warp's query (QPW == 1) as BF16 into shared memory, zeros for the chunk's missing queries
+    const bool have = warp < nq && nk[0] > 0;
+    const float inv = have ? 1.f / den[0] : 0.f;
 #pragma unroll
-  for (int t = 0; t < QPW; ++t) {
-    const int r = warp + ATT_WARPS * t;
-    if (r < nq && nk[t] > 0) {
-      const float inv = 1.f / den[t];
+    for (int rr = 0; rr < R; ++rr) a_s[warp][lane + 32 * rr] = __float2bfloat16_rn(have ? acc[0][rr] * inv : 0.f);
+    __syncthreads();
+    const int g = lane >> 2, t4 = lane & 3;
+    const int nrgw = d >> 7;
+    // B fragments: query g, K elements 8 t .. 8 t + 7 of each 32-wide chunk
+    const uint4 xb0 = *reinterpret_cast<const uint4*>(&a_s[g][8 * t4]);
+    const uint4 xb1 = *reinterpret_cast<const uint4*>(&a_s[g][32 + 8 * t4]);
+    float* obase = p.o_part + (size_t)h * p.o_stride + (size_t)m0 * d;
+    for (int r0 = 0; r0 < nrgw; r0 += 4) {
+      if (r0 > 0) {                                         // wider models: the next four row groups
+        const bf16* wbase = p.wo + (size_t)((warp * nrgw + r0) * 16 + g) * d + h * DH + 8 * t4;
 #pragma unroll
-      for (int rr = 0; rr < R; ++rr)
-        out[(size_t)(m0 + r) * d + h * DH + lane + 32 * rr] = from_f32<ActT>(acc[t][rr] * inv);
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            if (r0 + r < nrgw) {
+              wf[r][c][0] = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(r * 16) * d + c * 32));
+              wf[r][c][1] = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(r * 16 + 8) * d + c * 32));
+            }
+          }
+      }
+      float o[4][4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) { o[r][0] = 0.f; o[r][1] = 0.f; o[r][2] = 0.f; o[r][3] = 0.f; }
+      // the four MMAs of a row group share an accumulator: walk the groups in the inner loop so that dependent
+      // MMAs are four instructions apart
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const uint4 xb = c == 0 ? xb0 : xb1;
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          if (r0 + r < nrgw) att_mma_bf16(o[r], wf[r][c][0].x, wf[r][c][1].x, wf[r][c][0].y, wf[r][c][1].y, xb.x, xb.y);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          if (r0 + r < nrgw) att_mma_bf16(o[r], wf[r][c][0].z, wf[r][c][1].z, wf[r][c][0].w, wf[r][c][1].w, xb.z, xb.w);
+      }
+      // o[r]: features n, n + 8 (n = first feature of the group + g) of queries 2 t, 2 t + 1
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        if (r0 + r < nrgw) {
+          const int n = (warp * nrgw + r0 + r) * 16 + g;
+          const int q0 = 2 * t4, q1 = q0 + 1;
+          if (q0 < nq) { obase[(size_t)q0 * d + n] = o[r][0]; obase[(size_t)q0 * d + n + 8] = o[r][2]; }
+          if (q1 < nq) { obase[(size_t)q1 * d + n] = o[r][1]; obase[(size_t)q1 * d + n + 8] = o[r][3]; }
+        }
+      }
+    }
+  } else {
+    ActT* out = reinterpret_cast<ActT*>(p.out);
+#pragma unroll
+    for (int t = 0; t < QPW; ++t) {
+      const int r = warp + ATT_WARPS * t;
+      if (r < nq && nk[t] > 0) {
+        const float inv = 1.f / den[t];
+#pragma unroll
+        for (int rr = 0; rr < R; ++rr)
+          out[(size_t)(m0 + r) * d + h * DH + lane + 32 * rr] = from_f32<ActT>(acc[t][rr] * inv);
+      }
     }
   }
   trace_mark(TR_ATTN, 2);
