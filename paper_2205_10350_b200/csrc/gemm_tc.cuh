@@ -284,8 +284,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const bool early = (blockIdx.y == 0);   // token tile 0 always has work (M >= 1 whenever a result is read)
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
+  // MMA issuers.  Issuing one tcgen05.mma costs its thread 65-80 cycles whatever the tile, so with few tokens (short
+  // MMAs) a single issuer, not the tensor pipe or shared memory, sets the pace of the K loop.  Up to four threads in
+  // different warps therefore issue side by side: issuer j takes the K blocks j, j + n, j + 2n, ... of this CTA and
+  // accumulates them in its own ntile-column region of tensor memory; the epilogue adds the regions up.
+  // An issuer waits for ring phase r of a stage only after phase r - 1 has completed (a parity wait two phases ahead
+  // would alias): with more than one ring round this holds when the ring depth is a multiple of the issuer count, since
+  // the K block that used the stage one round earlier was then this issuer's own.
+  int n_issuers = 1;
+  {
+    const int cap = ntile <= 64 ? 4 : (ntile <= 128 ? 2 : 1);
+    for (int cand = 4; cand > 1; cand >>= 1)
+      if (cand <= cap && cand <= num_kb && (num_kb <= stages || stages % cand == 0)) { n_issuers = cand; break; }
+  }
   uint32_t tmem_cols = 32;
-  while (tmem_cols < (uint32_t)ntile) tmem_cols <<= 1;
+  while (tmem_cols < (uint32_t)(ntile * n_issuers)) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
@@ -294,7 +307,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
-    mbar_init(smem_u32(&bar_acc), 1);
+    mbar_init(smem_u32(&bar_acc), (uint32_t)n_issuers);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -367,52 +380,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         tma_load_2d(a_dst + A_STAGE_BYTES, &map_x, (kb_begin + i) * BLOCK_K, t0, bar);
       }
       if (warp == 0) trace_mark(TR_GEMM + EPI, 3);
-    } else if (warp == 1 && lane == 0) {
-      // ---- MMA issuer ----
-      // This single thread's instruction latencies add up once per K block, so the loop carries running stage /
-      // parity / descriptor values instead of recomputing them (no integer division, no address rebuilding).
+    } else if (warp >= 4 && warp - 4 < n_issuers && lane == 0) {
+      // ---- MMA issuers (lane 0 of warps 4 .. 4 + n_issuers - 1) ----
+      const int j = warp - 4;
       const uint32_t idesc = make_idesc(BLOCK_N_FEAT, ntile);
-      bool ok = true;
-      int s = 0;
-      uint32_t parity = 0;
+      const uint32_t acc_j = tmem_acc + (uint32_t)(j * ntile);
       const uint64_t desc_a0 = make_smem_desc(smem_base);
       const uint64_t desc_b0 = make_smem_desc(smem_base + A_STAGE_BYTES);
       const uint64_t desc_step = (uint64_t)(stage_bytes >> 4);     // stage stride in the (address >> 4) field
-      uint64_t desc_a = desc_a0, desc_b = desc_b0;
-      uint32_t bar_f = smem_u32(&bar_full[0]), bar_e = smem_u32(&bar_empty[0]);
-      // A barrier wait costs this thread ~0.14 us even when the phase completed long ago, so after every blocking
-      // wait the remaining stages of the ring round are probed in one batch (their latencies overlap) and the
-      // stages found complete are consumed without waiting again.
-      uint32_t ready_mask = 0;
-      for (int i = 0; i < num_kb; ++i) {
-        if (!((ready_mask >> s) & 1u)) {
-          ok = mbar_wait(bar_f, parity, p.status);
-          if (!ok) { abort_flag = 1; break; }
-          const int left = min(stages - s, num_kb - i);      // stages of this round from s on (s included)
-          uint32_t probe[MAX_STAGES];
-#pragma unroll
-          for (int t = 1; t < MAX_STAGES; ++t) probe[t] = (t < left) ? mbar_test(bar_f + 8 * t, parity) : 0u;
-#pragma unroll
-          for (int t = 1; t < MAX_STAGES; ++t) ready_mask |= probe[t] << ((s + t) & 31);
-        }
+      bool ok = true;
+      int s = j % stages;
+      uint32_t parity = (uint32_t)(j / stages) & 1u;
+      for (int i = j; i < num_kb; i += n_issuers) {
+        ok = mbar_wait(smem_u32(&bar_full[s]), parity, p.status);
+        if (!ok) { abort_flag = 1; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t desc_a = desc_a0 + desc_step * (uint64_t)s, desc_b = desc_b0 + desc_step * (uint64_t)s;
 #pragma unroll
         for (int k4 = 0; k4 < BLOCK_K / UMMA_K; ++k4) {
           // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the (address >> 4) field
-          umma_bf16(tmem_acc, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (i | k4) != 0 ? 1u : 0u);
+          umma_bf16(acc_j, desc_a + 2 * k4, desc_b + 2 * k4, idesc, (i != j || k4 != 0) ? 1u : 0u);
         }
         // the stage is handed back to the producers only if a later K block will land in it
-        if (i + stages < num_kb) umma_commit(bar_e);
-        if (++s == stages) {
-          s = 0; parity ^= 1; ready_mask = 0;
-          desc_a = desc_a0; desc_b = desc_b0;
-          bar_f = smem_u32(&bar_full[0]); bar_e = smem_u32(&bar_empty[0]);
-        } else {
-          desc_a += desc_step; desc_b += desc_step;
-          bar_f += 8; bar_e += 8;
-        }
+        if (i + stages < num_kb) umma_commit(smem_u32(&bar_empty[s]));
+        s += n_issuers;
+        while (s >= stages) { s -= stages; parity ^= 1u; }
       }
-      if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
+      // one arrival per issuer: the accumulator barrier fires when every region is complete.  An issuer that gave
+      // up still arrives (plainly), so that nobody waits for it; the abort flag tells the epilogue to do nothing.
+      if (ok) umma_commit(smem_u32(&bar_acc));
+      else asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_acc)) : "memory");
     }
     __syncwarp();
 
@@ -441,6 +438,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int c = grp * 16; c < ntile && c < ntok_all; c += 32) {
           float acc[16];
           tmem_ld16(tlane + static_cast<uint32_t>(c), acc);
+          for (int r = 1; r < n_issuers; ++r) {              // the other issuers' shares of the K range
+            float more[16];
+            tmem_ld16(tlane + static_cast<uint32_t>(r * ntile + c), more);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[j] += more[j];
+          }
           // columns past the last valid token hold whatever the padded activation rows produced: never stored
 #pragma unroll
           for (int j = 0; j < 16; ++j) acc[j] = n < p.N ? acc[j] + bias_n : -INFINITY;
@@ -493,6 +496,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       for (int c = grp * 16; c < sub && c < ntok; c += 32) {
         float acc[16];
         tmem_ld16(tlane + static_cast<uint32_t>(tb + c), acc);
+        for (int r = 1; r < n_issuers; ++r) {
+          float more[16];
+          tmem_ld16(tlane + static_cast<uint32_t>(r * ntile + tb + c), more);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) acc[j] += more[j];
+        }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           if (c + j < ntok) {
