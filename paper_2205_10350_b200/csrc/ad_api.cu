@@ -491,7 +491,7 @@ int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, co
   const size_t stride = (size_t)pc.M_cap * d;
   h->launches++;
   cudaError_t e;
-  if (pc.M_cap >= 512 && d % 128 == 0 && d <= 1024) {   // many tokens: a warp per token
+  if (pc.M_cap >= 512 && nsplit <= 4 && d % 128 == 0 && d <= 1024) {   // many tokens: a warp per token
     dim3 rgrid((pc.M_cap + 7) / 8);
     if (h->bf16) e = launch_k(layernorm_rows_kernel<bf16>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                               (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);

@@ -373,9 +373,11 @@ layernorm_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, i
 }
 
 // The same operation for large token counts: one warp per token (no block-wide barrier), 8 tokens per CTA.
+// The loads of two element groups (residual and up to four partial sums each: ten 16-byte loads per lane) are issued
+// before their first use.  nsplit <= 4 here (more partials take the one-CTA-per-token kernel).
 // grid = ceil(M_cap / 8), block = 256, d <= 1024 and a multiple of 128.
 template <typename ActT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 layernorm_rows_kernel(const int* __restrict__ M_ptr, const float* __restrict__ pre, int nsplit, size_t split_stride,
                       const float* __restrict__ bias, const float* resid, const float* __restrict__ g,
                       const float* __restrict__ bta, int d, float eps, float* y, ActT* __restrict__ yb) {
@@ -384,9 +386,6 @@ layernorm_rows_kernel(const int* __restrict__ M_ptr, const float* __restrict__ p
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int per = d >> 7;                               // float4 groups per lane (d / 128), <= 8
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
-  float4 cb[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) cb[i] = (i < per && bias) ? reinterpret_cast<const float4*>(bias)[lane + 32 * i] : zero4;
   pdl_wait();
   trace_mark(TR_LN, 1);
   const int m = blockIdx.x * 8 + warp;
@@ -395,19 +394,29 @@ layernorm_rows_kernel(const int* __restrict__ M_ptr, const float* __restrict__ p
     float4 xv[8];
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float4 v = zero4;
-      if (i < per) {
-        const size_t off = row + lane + 32 * i;
-        v = resid ? reinterpret_cast<const float4*>(resid)[off] : zero4;
-        v.x += cb[i].x; v.y += cb[i].y; v.z += cb[i].z; v.w += cb[i].w;
-        for (int sp = 0; sp < nsplit; ++sp) {
-          const float4 q = reinterpret_cast<const float4*>(pre + sp * split_stride)[off];
-          v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
-        }
+    for (int pair = 0; pair < 4; ++pair) {
+      if (pair * 2 >= per) break;
+      float4 r4[2], c4[2], q4[2][4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int gi = pair * 2 + i;
+        const size_t off = row + lane + 32 * gi;
+        r4[i] = (gi < per && resid) ? reinterpret_cast<const float4*>(resid)[off] : zero4;
+        c4[i] = (gi < per && bias) ? reinterpret_cast<const float4*>(bias)[lane + 32 * gi] : zero4;
+#pragma unroll
+        for (int sp = 0; sp < 4; ++sp)
+          q4[i][sp] = (gi < per && sp < nsplit) ? reinterpret_cast<const float4*>(pre + sp * split_stride)[off] : zero4;
       }
-      xv[i] = v;
-      s += v.x + v.y + v.z + v.w;
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int gi = pair * 2 + i;
+        float4 v = r4[i];
+        v.x += c4[i].x; v.y += c4[i].y; v.z += c4[i].z; v.w += c4[i].w;
+#pragma unroll
+        for (int sp = 0; sp < 4; ++sp) { v.x += q4[i][sp].x; v.y += q4[i][sp].y; v.z += q4[i][sp].z; v.w += q4[i][sp].w; }
+        xv[gi] = v;
+        s += v.x + v.y + v.z + v.w;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
