@@ -33,9 +33,12 @@ def test_fp32_linear(M, K, N):
 
 
 @pytest.mark.parametrize("M,K,N", [(1, 64, 128), (16, 64, 128), (64, 512, 1536), (25, 1024, 300), (200, 512, 512),
-                                   (256, 2048, 640), (7, 4096, 128)])
+                                   (256, 2048, 640), (7, 4096, 128), (100, 2048, 384), (100, 192, 256),
+                                   (12, 320, 20000)])
 def test_bf16_tensor_core_linear(M, K, N):
-    """Inputs are BF16-exact, the accumulator is FP32: only the summation order differs from the checker."""
+    """Inputs are BF16-exact, the accumulator is FP32: only the summation order differs from the checker.
+    The shapes walk through the kernel's configurations: one, two and four MMA issuers, K loops of one and of
+    several ring rounds, one and two CTAs per SM, ragged token and feature tiles."""
     x, W, b = _data(M, K, N, True)
     st = torch.zeros(1, dtype=torch.int32, device=DEV)
     y = binding.linear(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(W, device=DEV).bfloat16(),
