@@ -73,6 +73,13 @@ struct PassCfg {
   }
 };
 
+// A second set of activation buffers (encoder-pass sized) for work that runs on the side stream.
+struct ActSet {
+  float *y = nullptr, *pre = nullptr, *pre2 = nullptr;
+  ActBuf yb, abuf, hbuf;
+  void *qbuf = nullptr, *ktmp = nullptr, *vtmp = nullptr;
+};
+
 thread_local std::string g_create_error;
 
 }  // namespace
@@ -97,6 +104,10 @@ struct ad_handle {
   int* part_cnt = nullptr;   // relaxed verification: per tile and token, other tokens scoring above the draft
   float* draft_val = nullptr;
   int* draft_id = nullptr;
+  // The drafter's encoder does not depend on the verifier's: it runs on a side stream with its own activations.
+  ActSet side;
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int beta = 0;              // 0: exact-match verification; >= 1: relaxed verification (Section 3.2.3)
   float tau = 0.f;
   int n_vtiles = 0;
@@ -240,6 +251,19 @@ size_t layout(ad_handle* h, void* base) {
     h->nar.kenc = bp.take(cross_sz);
     h->nar.venc = bp.take(cross_sz);
   }
+  if (c.has_drafter) {
+    const int Me = h->pass[PK_ENCODE].M_cap;
+    ActSet& sd = h->side;
+    sd.y = (float*)bp.take(sizeof(float) * (size_t)Me * d);
+    sd.pre = (float*)bp.take(sizeof(float) * (size_t)h->pass[PK_ENCODE].max_split * Me * d);
+    if (h->bf16 && c.n_heads <= 16) sd.pre2 = (float*)bp.take(sizeof(float) * (size_t)c.n_heads * Me * d);
+    sd.yb.ptr = bp.take(e * (size_t)Me * d); sd.yb.cols = d;
+    sd.abuf.ptr = bp.take(e * (size_t)Me * d); sd.abuf.cols = d;
+    sd.hbuf.ptr = bp.take(e * (size_t)Me * F); sd.hbuf.cols = F;
+    sd.qbuf = bp.take(e * (size_t)Me * d);
+    sd.ktmp = bp.take(e * (size_t)Me * d);
+    sd.vtmp = bp.take(e * (size_t)Me * d);
+  }
   h->n_vtiles = (c.vocab + 127) / 128;
   h->part_val = (float*)bp.take(sizeof(float) * (size_t)h->n_vtiles * Mv);
   h->part_idx = (int*)bp.take(sizeof(int) * (size_t)h->n_vtiles * Mv);
@@ -325,6 +349,7 @@ int bind_model(ad_handle* h, Model& m, const ad_model_weights& w) {
 
 bool g_use_pdl = true;       // AD_NO_PDL=1 in the environment turns programmatic dependent launch off
 bool g_use_graph_encode = true;   // AD_NO_ENCODE_GRAPH=1: launch the encoder kernels directly
+bool g_two_stream_encode = true;   // AD_NO_CONCURRENT_ENCODERS=1: the drafter's encoder after the verifier's, on one stream
 bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
 bool g_fuse_attn_proj = true;   // AD_NO_ATTN_PROJ=1: attention and its output projection always as separate kernels
 
@@ -622,6 +647,15 @@ int encoder_pass(ad_handle* h, Model& m, bool keep_memory) {
   return AD_OK;
 }
 
+// Exchanges the handle's activation buffers and stream with the side set (and back, when called again).
+void swap_side(ad_handle* h) {
+  ActSet& sd = h->side;
+  std::swap(h->y, sd.y); std::swap(h->pre, sd.pre); std::swap(h->pre2, sd.pre2);
+  std::swap(h->yb, sd.yb); std::swap(h->abuf, sd.abuf); std::swap(h->hbuf, sd.hbuf);
+  std::swap(h->qbuf, sd.qbuf); std::swap(h->ktmp, sd.ktmp); std::swap(h->vtmp, sd.vtmp);
+  std::swap(h->stream, h->side_stream);
+}
+
 // Output projection fused with arg-max over X (yb for the verifier, the gathered mask rows for the drafter),
 // then the final reduction and (verifier) the draft compare.
 int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto_commit) {
@@ -755,6 +789,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   { const char* e = getenv("AD_NO_PDL"); g_use_pdl = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_DEVLOOP"); g_use_devloop = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ENCODE_GRAPH"); g_use_graph_encode = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_NO_CONCURRENT_ENCODERS"); g_two_stream_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ATTN_PROJ"); g_fuse_attn_proj = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
@@ -778,7 +813,21 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
         ok = ok && make_map(&b->map[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile);
         ok = ok && make_map(&b->map_half[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile / 2);
       }
+    if (cfg->has_drafter) {
+      const int Me = h->pass[PK_ENCODE].M_cap, nt = h->pass[PK_ENCODE].ntile;
+      ActBuf* sbufs[3] = {&h->side.yb, &h->side.abuf, &h->side.hbuf};
+      for (ActBuf* b : sbufs) {
+        ok = ok && make_map(&b->map[PK_ENCODE], b->ptr, Me, b->cols, nt);
+        ok = ok && make_map(&b->map_half[PK_ENCODE], b->ptr, Me, b->cols, nt / 2);
+      }
+    }
     if (!ok) return bail(AD_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  }
+  if (cfg->has_drafter && g_two_stream_encode) {
+    if (cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess)
+      return bail(AD_ERR_CUDA, "creating the side stream failed");
   }
   // Cache, scratch and state start from zero so that no stale bit pattern is ever read as a number.
   if (cudaMemsetAsync(workspace, 0, need, h->stream) != cudaSuccess) return bail(AD_ERR_CUDA, "clearing the workspace failed");
@@ -811,6 +860,9 @@ extern "C" int ad_destroy(ad_handle* h) {
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
   if (h->ev2) cudaEventDestroy(h->ev2);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->side_stream) { cudaStreamSynchronize(h->side_stream); cudaStreamDestroy(h->side_stream); }
   delete h;
   return AD_OK;
 }
@@ -851,6 +903,20 @@ extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, c
   auto enqueue = [&]() -> int {
     h->launches++;
     AD_CUDA(h, launch_k(plan_encode_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_ENCODE].plan, h->dims));
+    if (c.has_drafter && h->side_stream) {
+      // the two encoders are independent (Section 3.2: separate models): drafter's on the side stream, verifier's here
+      AD_CUDA(h, cudaEventRecord(h->ev_fork, h->stream));
+      AD_CUDA(h, cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+      swap_side(h);
+      const int rc_side = encoder_pass(h, h->nar, false);
+      cudaError_t e_join = rc_side == AD_OK ? cudaEventRecord(h->ev_join, h->stream) : cudaSuccess;
+      swap_side(h);
+      if (rc_side != AD_OK) return rc_side;
+      AD_CUDA(h, e_join);
+      AD_TRY(encoder_pass(h, h->ar, true));
+      AD_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_join, 0));
+      return AD_OK;
+    }
     AD_TRY(encoder_pass(h, h->ar, true));
     if (c.has_drafter) AD_TRY(encoder_pass(h, h->nar, false));
     return AD_OK;
