@@ -68,6 +68,27 @@ __device__ __forceinline__ void load8(const float* p, float* out) {
   out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
 }
 
+// Eight consecutive elements kept as loaded (no use of the data, so the load stays in flight) and widened later.
+template <typename T> struct Raw8;
+template <> struct Raw8<bf16> {
+  uint4 u;
+  __device__ __forceinline__ void load(const bf16* p) { u = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ void zero() { u = make_uint4(0u, 0u, 0u, 0u); }
+  __device__ __forceinline__ void widen(float* out) const {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { out[2 * t] = __uint_as_float(w[t] << 16); out[2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u); }
+  }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) { a = *reinterpret_cast<const float4*>(p); b = *reinterpret_cast<const float4*>(p + 4); }
+  __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+  __device__ __forceinline__ void widen(float* out) const {
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w; out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+  }
+};
+
 constexpr int ATT_WARPS = 8;   // warps per CTA
 constexpr int ATT_MAX_QSPLIT = 16;   // most split-K partials a query may be summed from
 constexpr int ATT_KT = 64;     // keys per shared-memory tile
@@ -81,7 +102,8 @@ constexpr size_t att_smem_bytes() {
 // row and one head and stages every K/V tile once for all of them).  QPW = 1 keeps the critical path short when
 // there are few queries; QPW = 8 amortises the K/V staging when there are thousands.
 // Global-memory round trips on the critical path: (1) the row's segment / key-range descriptors,
-// (2) the queries, their key counts and the first K/V tile together, then compute and store.
+// (2) the queries, their key counts and the first K/V tile together (the tile's loads are issued first and only
+// widened once the queries are in shared memory), then compute and store.
 // FUSE (BF16, 64-wide heads, one query per warp): the output projection of the 8 queries is done here as well (see
 // AttnParams::wo).  Warp w owns output features [w d / 8, (w + 1) d / 8); its weight fragments -- 16 rows x 64 columns
 // per group of rows, read with 16-byte loads whose eight elements are consecutive in K (the contraction index is
@@ -136,6 +158,23 @@ attention_kernel(const AttnParams p) {
   const ActT* vv = reinterpret_cast<const ActT*>(p.v);
   const int d = p.d;
 
+  // first K/V tile: requested now, used after the queries have been staged
+  constexpr int NPRE = (ATT_KT * (DH / 8) + 255) / 256;
+  Raw8<ActT> kpre[NPRE], vpre[NPRE];
+#pragma unroll
+  for (int u = 0; u < NPRE; ++u) {
+    const int idx = tid + 256 * u;
+    const int j = idx / (DH / 8), c = (idx % (DH / 8)) * 8;
+    if (idx < ATT_KT * (DH / 8) && j < row_nk) {
+      const size_t off = (size_t)(kbase + j) * d + h * DH + c;
+      kpre[u].load(kk + off);
+      vpre[u].load(vv + off);
+    } else {
+      kpre[u].zero();
+      vpre[u].zero();
+    }
+  }
+
   // this warp's queries (warp, warp + 8, ...) and their visible-key counts
   int nk[QPW];
 #pragma unroll
@@ -175,7 +214,21 @@ attention_kernel(const AttnParams p) {
 
   for (int j0 = 0; j0 < row_nk; j0 += ATT_KT) {
     __syncthreads();   // previous tile fully consumed
-    for (int idx = tid; idx < ATT_KT * (DH / 8); idx += 256) {
+    if (j0 == 0) {
+#pragma unroll
+      for (int u = 0; u < NPRE; ++u) {
+        const int idx = tid + 256 * u;
+        if (idx < ATT_KT * (DH / 8)) {
+          const int j = idx / (DH / 8), c = (idx % (DH / 8)) * 8;
+          float kf[8], vf[8];
+          kpre[u].widen(kf);
+          vpre[u].widen(vf);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) { ks[j][c + t] = kf[t]; vs[j][c + t] = vf[t]; }
+        }
+      }
+    }
+    for (int idx = tid; j0 > 0 && idx < ATT_KT * (DH / 8); idx += 256) {
       const int j = idx / (DH / 8), c = (idx % (DH / 8)) * 8;
       float kf[8], vf[8];
       if (j0 + j < row_nk) {
