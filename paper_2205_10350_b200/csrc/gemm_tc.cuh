@@ -7,10 +7,11 @@
 // Both operands are K-major (row-major [rows, K]) and land in shared memory in the 128-byte-swizzled
 // canonical layout that the TMA and the MMA shared-memory descriptor agree on.
 //
-// Thread roles inside the 256-thread CTA: lane 0 of several warps issues TMA loads, lane 0 of warp 1 issues the
-// MMAs, then all eight warps take part in the epilogue: warp w reads the 32 TMEM lanes of quadrant w % 4
-// (tcgen05.ld 32x32b) and the two warps of a quadrant share its token columns.  The epilogue is a chain of
-// dependent instructions per thread, so halving each thread's share of it shortens the kernel.
+// Thread roles inside the 256-thread CTA: lane 0 of several warps issues TMA loads, lane 0 of warps 4..7 issues the
+// MMAs (up to four issuers, each with its own accumulator region in tensor memory), then all eight warps take part
+// in the epilogue: warp w reads the 32 TMEM lanes of quadrant w % 4 (tcgen05.ld 32x32b), adds the issuers' regions
+// up, and the two warps of a quadrant share its token columns.  The epilogue is a chain of dependent instructions
+// per thread, so halving each thread's share of it shortens the kernel.
 // Every mbarrier wait is bounded; on expiry the kernel latches AD_ERR_TIMEOUT, frees its TMEM and returns.
 #pragma once
 
@@ -327,7 +328,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   // TMA issue is spread over lane 0 of all eight warps: one thread's bulk-tensor copies are processed one after
   // the other, several threads' copies run side by side.  Stage i of the first ring round belongs to warp i;
-  // later rounds are fed by warps 0, 2 and 3 (warp 1's lane 0 is busy issuing MMAs).
+  // later rounds are fed by warps 0, 2 and 3.
   if (early && lane == 0) {
     // weights never change: fetch the first ring round before the previous kernel has finished
     for (int i = warp; i < first_round; i += THREADS / 32) {
