@@ -155,3 +155,34 @@ def test_results_are_bit_reproducible_and_independent_of_the_block_partition():
     block = runs[0].reshape(2, 6, -1)              # rows packed row-major
     for b in range(2):
         assert np.abs(block[b] - single[:, b]).max() < 1e-5
+
+
+def test_encoders_on_two_streams_equal_encoders_in_sequence(monkeypatch):
+    """The drafter's encoder runs on a side stream next to the verifier's.  The same handle configuration with the
+    two passes in sequence on one stream (AD_NO_CONCURRENT_ENCODERS=1, read when the handle is created) must give the
+    same drafts, the same verified tokens and the same encoder memory, bit for bit."""
+    shape = synth.MINI_BF16
+    w, wn = synth.make_weights(shape, 0), synth.make_weights(shape, 1)
+    r = np.random.default_rng(41)
+    src = r.integers(4, shape.vocab, size=(3, 14)).astype(np.int32)
+    lens = np.array([14, 9, 11], np.int32)
+    got = []
+    for sequential in (False, True):
+        if sequential:
+            monkeypatch.setenv("AD_NO_CONCURRENT_ENCODERS", "1")
+        dec = binding.AggressiveDecoder(shape, w, wn, max_batch=3, max_src=14, max_tgt=16, kmax=6)
+        res = []
+        for _ in range(2):                      # second call replays the captured encode graph
+            dec.encode(src, lens)
+            mem = dec.debug_encoder_memory(1, int(lens[1]))
+            drafts, k = dec.draft_block(6)
+            ids, n = dec.verify_block(drafts, k)
+            res.append((mem, drafts, k, ids, n))
+        outs, _ = dec.generate(src, lens, mode="GAD", k=6, max_len=[12, 12, 12], run_drafter=True)
+        got.append((res, outs))
+        dec.close()
+    for (a, b) in zip(got[0][0], got[1][0]):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+    for x, y in zip(got[0][1], got[1][1]):
+        assert np.array_equal(x, y)
