@@ -318,9 +318,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  trace_mark(TR_GEMM + EPI, 6);
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  trace_mark(TR_GEMM + EPI, 7);
   const uint32_t tmem_acc = tmem_base_slot;
   // Successors may start now: this CTA already owns its tensor memory, so a later kernel's allocation can
   // never starve it.
@@ -417,7 +419,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // ---- epilogue: all eight warps ----
     bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     if (*reinterpret_cast<volatile int*>(&abort_flag)) ready = false;
-    ready = __syncthreads_and(ready) != 0;     // one verdict for the CTA (also makes slot_s visible)
+    ready = __syncthreads_and(ready) != 0;     // one decision for the CTA (also makes slot_s visible)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     trace_mark(TR_GEMM + EPI, 4);
     // The accumulator holds one output feature per TMEM lane and one token per column.  Warp w reads lanes
