@@ -12,6 +12,15 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu)")
 
 
+def pytest_sessionstart(session):
+    """A fresh checkout has no built library: compile it (nvcc cross-compiles without a GPU) when it is missing or older
+    than its sources.  Without nvcc the tests that need the library fail loudly, as the library's loader does."""
+    import shutil
+    from paper_2205_10350_b200 import build as b
+    if os.path.exists(os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")) or shutil.which("nvcc"):
+        b.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
