@@ -160,6 +160,13 @@ def run_reference(args, rank, world):
 # ------------------------------------------------------------------------------------------------------
 def run_ours(args, rank, world, local_rank):
     import torch
+    from paper_2205_10350_b200 import build as lib_build
+    if rank == 0:
+        lib_build.build()      # no-op when the in-tree library is newer than its sources
+    else:                      # the other ranks of a node wait for rank 0's build
+        t_wait = time.time()
+        while lib_build._stale() and time.time() - t_wait < 600:
+            time.sleep(1.0)
     from paper_2205_10350_b200 import binding
 
     dist = None
