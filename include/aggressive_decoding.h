@@ -132,7 +132,10 @@ int ad_query_workspace(const ad_model_cfg* cfg, size_t* bytes);
 /* Problem statement: "given model parameters Phi" (Algorithm 1, input line; Section 3.2).
  * Builds a handle over borrowed weights and workspace (device, >= ad_query_workspace bytes, 1024-byte
  * aligned).  `stream` is a cudaStream_t (NULL = default stream).  Computes the positional table on the
- * host and uploads it; encodes TMA descriptors for every weight matrix.  Synchronises the stream. */
+ * host and uploads it; encodes TMA descriptors for every weight matrix; copies the decoder layers' cross-attention
+ * key/value projection matrices and biases into the workspace as one matrix (ad_encode then projects the encoder
+ * memory for all layers in one launch), so a later change of those weights needs a new handle.  Synchronises the
+ * stream. */
 int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* workspace, size_t workspace_bytes,
               void* stream, ad_handle** out);
 int ad_destroy(ad_handle* h);

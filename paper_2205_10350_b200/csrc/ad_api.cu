@@ -49,6 +49,11 @@ struct Model {
   std::vector<DecLayer> dec;
   void* kenc = nullptr;   // [n_dec][B * max_src][d] cross-attention keys
   void* venc = nullptr;
+  // the decoder layers' cross-attention key/value projections gathered into one [n_dec * 2d, d] matrix (and their
+  // biases into one vector) at ad_create, so that ad_encode projects the encoder memory for all layers in one launch
+  Mat ckv_all;
+  void* ckv_pack = nullptr;
+  float* cbkv_pack = nullptr;
 };
 struct PassCfg {
   int M_cap = 0;     // packed-token capacity of this pass kind
@@ -263,6 +268,11 @@ size_t layout(ad_handle* h, void* base) {
     sd.qbuf = bp.take(e * (size_t)Me * d);
     sd.ktmp = bp.take(e * (size_t)Me * d);
     sd.vtmp = bp.take(e * (size_t)Me * d);
+  }
+  {
+    const size_t pack = e * (size_t)c.n_dec * 2 * d * d, bpack = sizeof(float) * (size_t)c.n_dec * 2 * d;
+    h->ar.ckv_pack = bp.take(pack); h->ar.cbkv_pack = (float*)bp.take(bpack);
+    if (c.has_drafter) { h->nar.ckv_pack = bp.take(pack); h->nar.cbkv_pack = (float*)bp.take(bpack); }
   }
   h->n_vtiles = (c.vocab + 127) / 128;
   h->part_val = (float*)bp.take(sizeof(float) * (size_t)h->n_vtiles * Mv);
@@ -637,13 +647,11 @@ int encoder_pass(ad_handle* h, Model& m, bool keep_memory) {
   }
   if (keep_memory)
     AD_CUDA(h, cudaMemcpyAsync(h->encmem, h->yb.ptr, (size_t)pc.M_cap * c.d_model * h->esz, cudaMemcpyDeviceToDevice, h->stream));
-  for (int l = 0; l < c.n_dec; ++l) {
-    DecLayer& L = m.dec[l];
-    GemmParams p = {};
-    p.bias = L.cbkv; p.dst[0] = (char*)m.kenc + l * cross_layer; p.dst[1] = (char*)m.venc + l * cross_layer;
-    p.seg_width = c.d_model; p.n_direct = 0; p.slot = h->st.enc_slot;
-    AD_TRY(gemm(h, EPI_SCATTER, L.ckv, h->yb, PK_ENCODE, pc.plan.M, pc.M_cap, p));
-  }
+  // cross-attention keys and values of every decoder layer in one launch (segments 2l / 2l + 1 = layer l's K / V)
+  GemmParams p = {};
+  p.bias = m.cbkv_pack; p.dst[0] = m.kenc; p.dst[1] = m.venc; p.seg_pair_stride = cross_layer;
+  p.seg_width = c.d_model; p.n_direct = 0; p.slot = h->st.enc_slot;
+  AD_TRY(gemm(h, EPI_SCATTER, m.ckv_all, h->yb, PK_ENCODE, pc.plan.M, pc.M_cap, p));
   return AD_OK;
 }
 
@@ -831,6 +839,20 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   }
   // Cache, scratch and state start from zero so that no stale bit pattern is ever read as a number.
   if (cudaMemsetAsync(workspace, 0, need, h->stream) != cudaSuccess) return bail(AD_ERR_CUDA, "clearing the workspace failed");
+  // Gather the cross-attention key/value projections of all decoder layers (see Model::ckv_all).
+  for (Model* mp : {&h->ar, &h->nar}) {
+    if (!mp->present) continue;
+    const int d = cfg->d_model;
+    const size_t one = h->esz * (size_t)2 * d * d;
+    bool okc = true;
+    for (int l = 0; l < cfg->n_dec; ++l) {
+      okc = okc && cudaMemcpyAsync((char*)mp->ckv_pack + l * one, mp->dec[l].ckv.ptr, one, cudaMemcpyDeviceToDevice, h->stream) == cudaSuccess;
+      okc = okc && cudaMemcpyAsync(mp->cbkv_pack + (size_t)l * 2 * d, mp->dec[l].cbkv, sizeof(float) * 2 * d, cudaMemcpyDeviceToDevice, h->stream) == cudaSuccess;
+    }
+    mp->ckv_all.ptr = mp->ckv_pack; mp->ckv_all.N = cfg->n_dec * 2 * d; mp->ckv_all.K = d;
+    if (h->bf16) okc = okc && make_map(&mp->ckv_all.map, mp->ckv_pack, mp->ckv_all.N, d, tc::BLOCK_N_FEAT);
+    if (!okc) return bail(AD_ERR_CUDA, "gathering the cross-attention key/value projections failed");
+  }
   // Sinusoidal positional table PE(p, 2i) = sin(p / 10000^(2i/d)), PE(p, 2i+1) = cos(.), evaluated in double.
   {
     const int d = cfg->d_model;

@@ -44,7 +44,9 @@ enum Epi : int {
   EPI_F32 = 0,      // out_f32[m][n] = acc (+ bias) (+ resid[m][n])
   EPI_ACT = 1,      // out_act[m][n] = act(acc + bias), optional ReLU
   EPI_SCATTER = 2,  // feature n belongs to segment n / seg_width; segment s goes to dst[s] at row
-                    //   (s < n_direct ? m : slot[m]), column n % seg_width
+                    //   (s < n_direct ? m : slot[m]), column n % seg_width.  With seg_pair_stride != 0 there may be any
+                    //   number of segments: segment s goes to dst[s & 1] + (s >> 1) * seg_pair_stride bytes (key / value
+                    //   buffers of consecutive layers)
   EPI_ARGMAX = 3    // per (feature tile, token) running (max, lowest id) partials
 };
 
@@ -64,6 +66,7 @@ struct GemmParams {
   void* out_act;         // [M_cap, N] float or bf16
   // EPI_SCATTER
   void* dst[3];
+  size_t seg_pair_stride;
   int seg_width;
   int n_direct;
   const int* slot;       // [M_cap]

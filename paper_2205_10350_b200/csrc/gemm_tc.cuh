@@ -243,7 +243,9 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int n, int m
     } else if (EPI == EPI_SCATTER) {
       const int s = n / p.seg_width, c = n - s * p.seg_width;
       const int row = (s < p.n_direct) ? m : slot_s[j0 + j];
-      reinterpret_cast<ActT*>(p.dst[s])[(size_t)row * p.seg_width + c] = from_f32<ActT>(v);
+      char* seg_base = p.seg_pair_stride ? static_cast<char*>(p.dst[s & 1]) + (size_t)(s >> 1) * p.seg_pair_stride
+                                         : static_cast<char*>(p.dst[s]);
+      reinterpret_cast<ActT*>(seg_base)[(size_t)row * p.seg_width + c] = from_f32<ActT>(v);
     }
   }
 }
@@ -541,7 +543,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           width = p.seg_width;
           seg = n0 / width;
           col0 = n0 - seg * width;
-          base = reinterpret_cast<bf16*>(p.dst[seg]);
+          base = p.seg_pair_stride ? reinterpret_cast<bf16*>(static_cast<char*>(p.dst[seg & 1]) + (size_t)(seg >> 1) * p.seg_pair_stride)
+                                   : reinterpret_cast<bf16*>(p.dst[seg]);
         }
         const bool vec = (width & 7) == 0;
         for (int r = warp * 2 + half; r < ntok; r += THREADS / 16) {
