@@ -120,3 +120,52 @@ def check_free_run(out, greedy, margin, where=""):
     p = int(diff[0])
     assert margin[p] <= MARGIN, f"{where}: first difference at {p} where the checker's margin is {margin[p]:.3f}"
     return p
+
+
+def drafter_at_prefix(dec, nar_model, src, lens, prefixes, k, tol, exact=False):
+    """Draft substep at a NON-empty accepted prefix: walks every row of the library to the given prefix by teacher
+    forcing (verify + forced commit, in rounds of at most kmax tokens), then compares ad_draft_block with the checker's
+    drafter forward over (BOS, prefix, k x [MASK]): scores within tol, ids exact where the checker's top-1/top-2 gap
+    exceeds the margin (everywhere when exact), else one of the checker's top two.  Rows may have different prefix
+    lengths.  Returns the counts of exactly compared / ambiguous / flipped positions."""
+    B = len(lens)
+    dec.encode(src, lens)
+    done = [0] * B
+    while any(done[b] < len(prefixes[b]) for b in range(B)):
+        ks = np.zeros(B, np.int32)
+        toks = np.full((B, dec.kmax), -1, np.int32)
+        for b in range(B):
+            seg = np.asarray(prefixes[b][done[b]: done[b] + dec.kmax], np.int32)
+            ks[b] = len(seg)
+            toks[b, : len(seg)] = seg
+            done[b] += len(seg)
+        dec.verify_block(toks, ks)
+        dec.force_commit(toks, ks)
+    ln, _, _ = dec.state()
+    assert [int(x) for x in ln] == [len(p) for p in prefixes]
+    d, kk = dec.draft_block(k)
+    want_k = [min(k, dec.max_tgt - len(prefixes[b])) for b in range(B)]
+    assert [int(x) for x in kk] == want_k
+    scores = dec.debug_logits(int(sum(want_k)), which=1)
+    stats = dict(exact=0, ambiguous=0, flipped=0, worst=0.0)
+    off = 0
+    for b in range(B):
+        j, kb = len(prefixes[b]), want_k[b]
+        mem = nar_model.encode_memory(src[b, : lens[b]])
+        tokens = [nar_model.bos] + [int(t) for t in prefixes[b]]
+        ref_d, ref_m = nar_model.nar_draft(mem, tokens, kb)
+        ref_l = nar_model.decode_full(mem, np.array(tokens + [nar_model.mask] * kb, np.int32), causal=False)[j + 1:]
+        err = float(np.abs(scores[off: off + kb] - ref_l).max())
+        stats["worst"] = max(stats["worst"], err)
+        assert err <= tol, f"row {b}: drafter scores differ by {err:.3e} > {tol}"
+        for i in range(kb):
+            if exact or ref_m[i] > MARGIN:
+                assert d[b, i] == ref_d[i], f"row {b} slot {i}: draft {d[b, i]} != {ref_d[i]} at margin {ref_m[i]:.3f}"
+                stats["exact"] += 1
+            else:
+                stats["ambiguous"] += 1
+                if d[b, i] != ref_d[i]:
+                    stats["flipped"] += 1
+                    assert d[b, i] == second_best(ref_l[i], ref_d[i]), f"row {b} slot {i}: neither of the checker's top two"
+        off += kb
+    return stats

@@ -78,6 +78,37 @@ def test_tiny_generalized_mode_with_real_drafter(tiny):
         assert d[0, i] == ref_d[i] or ref_m[i] <= P.MARGIN
 
 
+def test_tiny_drafter_block_at_nonempty_prefix(tiny):
+    """Section 3.2.1: the drafter conditions on the accepted prefix.  FP32 model: ids identical to the checker's."""
+    dec, _, on = tiny
+    src, lens = synth.make_sources(synth.WORKLOADS[1])
+    r = np.random.default_rng(3)
+    for j, k in ((1, 5), (7, 17), (19, 9), (23, 4)):      # the last two are clipped by the remaining length
+        prefix = r.integers(4, synth.TINY.vocab, size=j)
+        st = P.drafter_at_prefix(dec, on, src, lens, [prefix], k, TOL_FP32, exact=True)
+        print(f"tiny drafter j={j} k={k}: {st}")
+
+
+def test_varied_fp32_drafter_ragged_prefixes():
+    """Three rows with different prefix lengths (one empty) through one drafter pass; larger weights so that the
+    prefix really changes the drafts."""
+    shape = synth.ModelShape("vary", 64, 2, 128, 40, 1, 2, "fp32")
+    dec, om, on = make(shape, 3, 12, 30, 13, drafter=True, std=0.15)
+    r = np.random.default_rng(6)
+    lens = np.array([12, 7, 9], np.int32)
+    src = np.full((3, 12), synth.PAD, np.int32)
+    for b in range(3):
+        src[b, : lens[b]] = r.integers(4, 40, size=lens[b])
+    prefixes = [r.integers(4, 40, size=n) for n in (14, 0, 5)]
+    st = P.drafter_at_prefix(dec, on, src, lens, prefixes, 6, TOL_FP32, exact=True)
+    print(f"varied drafter: {st}")
+    # the prefix matters: the same rows at an empty prefix draft something else somewhere
+    d0 = on.nar_draft(on.encode_memory(src[0, :12]), [0], 6)[0]
+    d1 = on.nar_draft(on.encode_memory(src[0, :12]), [0] + [int(t) for t in prefixes[0]], 6)[0]
+    assert not np.array_equal(d0, d1)
+    dec.close()
+
+
 # A model with larger weights decodes to varied text, which exercises suffix matching, rollback and EOS.
 @pytest.mark.parametrize("seed_std", [0.08, 0.15])
 def test_varied_fp32_model_all_modes(seed_std):
@@ -130,6 +161,11 @@ def test_mini_bf16_lockstep_and_generate():
     outs, _ = dec.generate(src, lens, mode="GAD", k=8, max_len=max_len, run_drafter=True)
     for b in range(4):
         P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"GAD row {b}")
+    # drafter at ragged non-empty prefixes (Section 3.2.1)
+    r = np.random.default_rng(12)
+    prefixes = [r.integers(4, shape.vocab, size=n) for n in (3, 11, 0, 17)]
+    st = P.drafter_at_prefix(dec, on, src, lens, prefixes, 8, TOL_BF16)
+    print(f"mini bf16 drafter at prefixes 3/11/0/17: {st}")
 
 
 # ------------------------------------------------------------------------------------------ workloads 2, 3
@@ -200,6 +236,8 @@ def test_workload4_big_generalized():
     greedy, streams = _greedy_streams(om, src, lens, max_len, wl.agreement, wl.index, wl.shape.vocab)
     dec.encode(src, lens)
     _drafter_parity(dec, on, src, lens, wl.k)
+    st = P.drafter_at_prefix(dec, on, src, lens, [greedy[0][0][:9]], wl.k, TOL_BF16)
+    print(f"big drafter at a 9-token prefix: {st}")
     tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, max_steps=3)
     assert tot["steps"] >= 1
     outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=max_len, draft_override=streams, run_drafter=True)

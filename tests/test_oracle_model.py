@@ -164,3 +164,89 @@ def test_zero_sublayers_make_the_choice_depend_on_the_last_token_only():
     st2 = m.state(np.array([40, 41, 42, 43, 44], np.int32))   # other source: must not matter
     b = st2.decode_block([0, 9, 9, 13])
     assert np.allclose(a, b, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------------
+# Pins of the drafter forward (Section 3.2 "Draft", Section 3.2.1): inputs (o_0..o_j, k x [MASK]) at positions
+# 0..j+k, bidirectional attention, drafts = greedy choices at the k mask positions.
+# ---------------------------------------------------------------------------------------------------
+def _ln(x, g, b, eps=1e-5):
+    mu = x.mean()
+    var = ((x - mu) ** 2).mean()
+    return (x - mu) / np.sqrt(var + eps) * g + b
+
+
+def _zero_sublayer_choice(w, shape, token, pos):
+    """Closed form of the decoder's greedy choice for one (token, position) when every projection and FFN matrix
+    is zero: each sublayer adds only its output bias to the residual before its LayerNorm."""
+    d = shape.d_model
+    x = np.asarray(w["emb"], np.float64)[token] * np.sqrt(d) + _pe(pos + 1, d)[pos]
+    for l in range(shape.n_dec):
+        p = f"dec.{l}"
+        x = _ln(x + w[f"{p}.self.o.b"], w[f"{p}.ln1.g"], w[f"{p}.ln1.b"])
+        x = _ln(x + w[f"{p}.cross.o.b"], w[f"{p}.ln2.g"], w[f"{p}.ln2.b"])
+        x = _ln(x + w[f"{p}.ffn2.b"], w[f"{p}.ln3.g"], w[f"{p}.ln3.b"])
+    logits = np.asarray(w["emb"], np.float64) @ x
+    order = np.argsort(-logits, kind="stable")
+    return int(order[0]), float(logits[order[0]] - logits[order[1]])
+
+
+def test_drafter_block_on_a_zero_sublayer_model_has_a_closed_form():
+    """With all matrices zero the drafter's choice at mask slot t is a function of ([MASK], position j+1+t) alone, which
+    is evaluated here directly; a drafter that fed [PAD], read the rows one off, or numbered the positions from the
+    block start instead of from 0 gives another id or another top-1/top-2 gap (checked below by evaluating those wrong
+    forms)."""
+    w = synth.make_weights(SHAPE, 3, std=0.3)
+    for name in w:
+        if name.endswith(".W"):
+            w[name] = np.zeros_like(w[name])
+    m = O.Model(SHAPE, w, max_pos=40, real="f64")
+    mem = m.encode_memory(np.array([5, 6, 7, 8], np.int32))
+    differs_pad = differs_shift = differs_origin = 0
+    for j, k in ((0, 5), (3, 4), (7, 9), (12, 1)):
+        prefix = [0] + [int(t) for t in np.random.default_rng(j).integers(4, SHAPE.vocab, size=j)]
+        draft, margin = m.nar_draft(mem, prefix, k)
+        for t in range(k):
+            want, gap = _zero_sublayer_choice(w, SHAPE, m.mask, j + 1 + t)
+            assert draft[t] == want, (j, k, t)
+            assert abs(margin[t] - gap) < 1e-9
+            other = lambda r: r[0] != want or abs(r[1] - gap) > 1e-6     # another id, or another top-1/top-2 gap
+            differs_pad += other(_zero_sublayer_choice(w, SHAPE, m.pad, j + 1 + t))
+            differs_shift += other(_zero_sublayer_choice(w, SHAPE, m.mask, j + t))
+            differs_origin += other(_zero_sublayer_choice(w, SHAPE, m.mask, t)) if j > 0 else 1
+    # the pin has teeth: each plausible mistake changes every one of the 19 (id, gap) pairs
+    assert differs_pad == 19 and differs_shift == 19 and differs_origin == 19
+
+
+@pytest.mark.parametrize("j,k", [(0, 4), (2, 3), (5, 6)])
+def test_drafter_block_matches_torch_nn_transformer_without_a_mask(weights, j, k):
+    """The full drafter forward (non-zero weights) against torch.nn's decoder layers run without a target mask over
+    (prefix, k x [MASK]): same ids at rows j+1 .. j+k, same top-1/top-2 gaps; and a causal run disagrees, so the
+    bidirectional attention is really exercised."""
+    src = np.array([7, 9, 4, 33, 21, 8], np.int32)
+    m = O.Model(SHAPE, weights, max_pos=32, real="f64")
+    mem = m.encode_memory(src)
+    prefix = [0] + [int(t) for t in np.random.default_rng(100 + j).integers(4, SHAPE.vocab, size=j)]
+    draft, margin = m.nar_draft(mem, prefix, k)
+
+    enc, dec = _torch_model(weights, SHAPE)
+    d = SHAPE.d_model
+    emb = torch.tensor(weights["emb"].astype(np.float64))
+    tok = np.array(prefix + [m.mask] * k)
+    with torch.no_grad():
+        x = (emb[torch.tensor(src, dtype=torch.long)] * np.sqrt(d) + torch.tensor(_pe(len(src), d))).unsqueeze(1)
+        for e in enc:
+            x = e(x)
+        outs = {}
+        for causal in (False, True):
+            y = (emb[torch.tensor(tok, dtype=torch.long)] * np.sqrt(d) + torch.tensor(_pe(len(tok), d))).unsqueeze(1)
+            mask = torch.nn.Transformer.generate_square_subsequent_mask(len(tok), dtype=torch.float64) if causal else None
+            for dl in dec:
+                y = dl(y, x, tgt_mask=mask)
+            outs[causal] = (y.squeeze(1) @ emb.T).numpy()
+    ref = outs[False][j + 1:]
+    assert np.array_equal(draft, ref.argmax(1))
+    top2 = np.sort(ref, axis=1)[:, -2:]
+    assert np.allclose(margin, top2[:, 1] - top2[:, 0], atol=1e-8)
+    if k > 1:      # earlier mask slots see later ones only when attention is bidirectional
+        assert np.abs(outs[True][j + 1:-1] - ref[:-1]).max() > 1e-6
