@@ -220,11 +220,23 @@ int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_
 /* Debug: FP32 copy of the verifier's encoder memory of row b, [src_len_b, d_model] (device pointer). */
 int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size_t capacity_elems);
 
-/* Debug: exercises the bounded-wait mechanism that every mbarrier wait of the GEMM kernels uses.  Launches one
- * tiny kernel that polls, at most poll_limit (1..65536) times, a barrier phase that nothing completes; the wait
- * runs out, AD_ERR_TIMEOUT is latched in *status (device int, must be 0 before) and the kernel returns
- * normally, leaving the context usable.  polls_done (device int, may be NULL) receives the number of polls. */
-int ad_debug_wait_probe(int32_t* status, int32_t poll_limit, int32_t* polls_done, void* stream);
+/* Debug: exercises the bounded-wait mechanism that every mbarrier wait of the GEMM kernels uses (a wait gives up
+ * after a time budget measured on the GPU's global timer: 20 ms in the kernels, budget_us here).  Launches one tiny
+ * kernel that waits, for at most budget_us (1..65536) microseconds, on a barrier phase that nothing completes; the
+ * wait runs out, AD_ERR_TIMEOUT is latched in *status (device int, must be 0 before) and the kernel returns
+ * normally, leaving the context usable.  waited_us (device int, may be NULL) receives the time the wait took. */
+int ad_debug_wait_probe(int32_t* status, int32_t budget_us, int32_t* waited_us, void* stream);
+
+/* Debug: self-test and timing of the grid-wide barrier the persistent decoder kernel is built on (a monotonically
+ * increasing arrival counter in global memory, release-add / acquire-poll, every wait bounded by time).  Launches,
+ * cooperatively, n_ctas CTAs (0 = one per SM) of 256 threads holding 160 KB of shared memory each; per round every CTA
+ * publishes a word, passes the barrier and checks the word of its neighbour.  absent_cta >= 0 names a CTA that leaves
+ * without arriving: the others' first wait then runs out after budget_us (1..65536), AD_ERR_TIMEOUT is latched in
+ * *status and the kernel returns normally.  scratch: device memory, 256-byte aligned, >= 256 + 8 * n_ctas bytes.
+ * result (device float[4]): [0] nanoseconds per barrier, [1] rounds completed, [2] payload mismatches (must be 0).
+ * Asynchronous on `stream`.  Errors: AD_ERR_ARG, AD_ERR_CAPACITY (more CTAs than fit at once), AD_ERR_CUDA. */
+int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32_t absent_cta, int32_t budget_us, void* scratch,
+                                size_t scratch_bytes, int32_t* status, float* result, void* stream);
 
 /* ---- single-kernel entry points (operator-level tests and microbenchmarks) --------------------------
  * All pointers are device pointers; `stream` is a cudaStream_t.  Asynchronous. */

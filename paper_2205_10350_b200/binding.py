@@ -22,7 +22,7 @@ EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
     "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync", "ad_set_acceptance",
     "ad_debug_logits", "ad_debug_encoder_memory", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
-    "ad_vocab_argmax_static", "ad_debug_wait_probe",
+    "ad_vocab_argmax_static", "ad_debug_wait_probe", "ad_debug_grid_barrier_probe",
     "ad_linear",
 ]
 
@@ -94,6 +94,7 @@ def load():
         "ad_vocab_argmax_static": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "ad_linear": (C.c_int, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "ad_debug_wait_probe": (C.c_int, [vp, i32, vp, vp]),
+        "ad_debug_grid_barrier_probe": (C.c_int, [i32, i32, i32, i32, vp, sz, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         f = getattr(lib, name)

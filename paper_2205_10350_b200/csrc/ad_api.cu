@@ -15,6 +15,7 @@
 #include "attention_mma.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "grid_sync.cuh"
 #include "steps.cuh"
 
 using namespace ad;
@@ -377,15 +378,22 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
+// Per-device caches (a process may hold handles on several GPUs): SM count, and which kernels already had their
+// dynamic shared-memory limit raised on that device (the attribute is per device, not per process).
+constexpr int kMaxDevices = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
 int num_sms() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
+  static int n[kMaxDevices] = {};
+  const int dev = current_device();
+  if (!n[dev]) {
+    cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (n[dev] <= 0) n[dev] = 148;
   }
-  return n;
+  return n[dev];
 }
 
 // Ring depth: as deep as ~200 KB of shared memory allows when the grid fits one wave; with more CTAs than SMs,
@@ -400,11 +408,12 @@ int tc_stages(int ntile, int kb, int n_ctas) {
 
 template <int EPI>
 cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const GemmParams& p, int M_cap) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};
+  const int dev = current_device();
+  if (!attr_set[dev]) {
     cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 204 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   const int ksplit = (EPI == EPI_F32 && p.ksplit > 1) ? p.ksplit : 1;
   dim3 grid((p.N + 127) / 128, (M_cap + p.ntile - 1) / p.ntile, ksplit);
@@ -451,12 +460,13 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
 template <typename T, int D, int Q, bool FUSE = false>
 cudaError_t launch_attention(dim3 grid, dim3 block, cudaStream_t st, const AttnParams& p) {
   constexpr size_t smem = att_smem_bytes<D, Q>();
-  static bool attr_set = false;
-  if (!attr_set && smem > 48 * 1024) {
+  static bool attr_set[kMaxDevices] = {};
+  const int dev = current_device();
+  if (!attr_set[dev] && smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  attr_set = true;
+  attr_set[dev] = true;
   return launch_k(attention_kernel<T, D, Q, FUSE>, grid, block, smem, st, p);
 }
 
@@ -809,7 +819,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   const size_t need = layout(h, workspace);
   auto bail = [&](int code, const std::string& msg) { g_create_error = msg; delete h; return code; };
   if (need > workspace_bytes) return bail(AD_ERR_CAPACITY, "workspace too small: need " + std::to_string(need) + " bytes");
-  h->dims = Dims{cfg->max_batch, cfg->max_src, cfg->max_tgt, cfg->kmax, cfg->bos, cfg->pad, cfg->eos, cfg->mask};
+  h->dims = Dims{cfg->max_batch, cfg->max_src, cfg->max_tgt, cfg->kmax, cfg->bos, cfg->pad, cfg->eos, cfg->mask, cfg->vocab};
   int rc = bind_model(h, h->ar, w->ar);
   if (rc == AD_OK && cfg->has_drafter) rc = bind_model(h, h->nar, w->nar);
   if (rc != AD_OK) return bail(rc, h->err);
@@ -1064,22 +1074,24 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
   if (opts->mode == AD_MODE_GAD && !opts->run_drafter && !opts->draft_override) return fail(h, AD_ERR_ARG, "GAD without the drafter needs draft_override");
   if (opts->draft_override && opts->override_stride < 1) return fail(h, AD_ERR_ARG, "override_stride must be positive");
   if (out_stride < 1) return fail(h, AD_ERR_ARG, "out_stride must be positive");
+  if (B < 1 || B > c.max_batch) return fail(h, AD_ERR_CAPACITY, "B outside 1..max_batch");
+  // host-visible per-row caps are checked before any device work, so a rejected call leaves the handle untouched
+  int max_iters = c.max_tgt;
+  if (opts->max_len && on_host) {
+    max_iters = 1;
+    for (int b = 0; b < B; ++b) {
+      if (opts->max_len[b] < 1 || opts->max_len[b] > c.max_tgt) return fail(h, AD_ERR_ARG, "max_len outside 1..max_tgt");
+      if (opts->max_len[b] > max_iters) max_iters = opts->max_len[b];
+    }
+  }
 
   AD_CUDA(h, cudaEventRecord(h->ev0, h->stream));
   h->launches = 0;
   AD_TRY(ad_encode(h, src, src_stride, src_len, B, on_host));
-  int max_iters = c.max_tgt;
   if (opts->max_len) {
     AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, opts->max_len, sizeof(int) * B, to_dev(on_host), h->stream));
     h->launches++;
     AD_CUDA(h, launch_k(set_maxlen_kernel, dim3((B + 63) / 64), dim3(64), 0, h->stream, h->st, h->dims, h->st.user_n));
-    if (on_host) {
-      max_iters = 1;
-      for (int b = 0; b < B; ++b) {
-        if (opts->max_len[b] < 1 || opts->max_len[b] > c.max_tgt) return fail(h, AD_ERR_ARG, "max_len outside 1..max_tgt");
-        if (opts->max_len[b] > max_iters) max_iters = opts->max_len[b];
-      }
-    }
   }
   const int* ovr = nullptr;
   int ovr_len = 0;   // valid leading entries of each staged override row
@@ -1247,25 +1259,94 @@ extern "C" int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size
 // ---- bounded-wait self-test ---------------------------------------------------------------------------
 
 namespace {
-// One thread waits, with the given poll limit, on an mbarrier phase that nothing ever completes.
-__global__ void wait_probe_kernel(int* status, unsigned int limit, int* polls_done) {
+// One thread waits, with the given time budget, on an mbarrier phase that nothing ever completes.
+__global__ void wait_probe_kernel(int* status, unsigned int budget_us, int* waited_us) {
   __shared__ __align__(8) uint64_t bar;
   if (threadIdx.x == 0) {
     tc::mbar_init(tc::smem_u32(&bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    unsigned int i = 0;
-    bool done = false;
-    for (; i < limit && !done; ++i) done = tc::mbar_try_wait(tc::smem_u32(&bar), 0);
-    if (!done) latch_error(status, AD_ERR_TIMEOUT);
-    if (polls_done) *polls_done = (int)i;
+    const unsigned long long t0 = tc::global_ns();
+    tc::mbar_wait_budget(tc::smem_u32(&bar), 0, status, (unsigned long long)budget_us * 1000ull);
+    if (waited_us) *waited_us = (int)((tc::global_ns() - t0) / 1000ull);
   }
 }
 }  // namespace
 
-extern "C" int ad_debug_wait_probe(int32_t* status, int32_t poll_limit, int32_t* polls_done, void* stream) {
-  if (!status || poll_limit < 1 || poll_limit > (1 << 16)) return AD_ERR_ARG;
-  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, (unsigned int)poll_limit, polls_done);
+extern "C" int ad_debug_wait_probe(int32_t* status, int32_t budget_us, int32_t* waited_us, void* stream) {
+  if (!status || budget_us < 1 || budget_us > (1 << 16)) return AD_ERR_ARG;
+  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, (unsigned int)budget_us, waited_us);
   return cudaGetLastError() == cudaSuccess ? AD_OK : AD_ERR_CUDA;
+}
+
+// ---- grid-barrier self-test and timing ------------------------------------------------------------------
+
+namespace {
+// Every CTA: per round, publish a word, pass the grid barrier, read the next CTA's word (bypassing L1) and check
+// it.  CTA `absent` (if any) leaves at once without ever arriving, so everybody else's first wait runs out.
+// result[0] = nanoseconds per barrier seen by CTA 0, result[1] = rounds CTA 0 completed, result[2] = payload
+// mismatches seen by any CTA (must be 0).
+__global__ void __launch_bounds__(256, 1)
+grid_barrier_probe_kernel(unsigned int* ctr, unsigned int* payload, int rounds, int absent, unsigned long long budget_ns,
+                          int* status, float* result) {
+  extern __shared__ uint8_t probe_smem[];    // only there to hold the SM: one CTA per SM, as in the persistent kernels
+  __shared__ int flag;
+  const unsigned int n = gridDim.x;
+  if ((int)blockIdx.x == absent) return;
+  unsigned int gen = 0;
+  int bad = 0, done = 0;
+  if (threadIdx.x == 0) probe_smem[0] = 0;
+  const unsigned long long t0 = gs::now_ns();
+  for (int r = 0; r < rounds; ++r) {
+    unsigned int* slot = payload + (size_t)(r & 1) * n;
+    if (threadIdx.x == 0) slot[blockIdx.x] = (unsigned int)r * 4096u + blockIdx.x;
+    if (!gs::grid_barrier(ctr, gen, n, budget_ns, &flag)) {
+      if (threadIdx.x == 0) latch_error(status, AD_ERR_TIMEOUT);
+      break;
+    }
+    const unsigned int nb = (blockIdx.x + 1) % n;
+    if (threadIdx.x == 0 && __ldcg(slot + nb) != (unsigned int)r * 4096u + nb) bad++;
+    ++done;
+  }
+  const unsigned long long t1 = gs::now_ns();
+  if (threadIdx.x == 0) {
+    if (bad) atomicAdd(reinterpret_cast<int*>(result + 2), bad);
+    if (blockIdx.x == (absent == 0 ? 1 : 0)) {
+      result[0] = done > 0 ? (float)(t1 - t0) / (float)done : 0.f;
+      result[1] = (float)done;
+    }
+  }
+}
+constexpr int kProbeSmem = 160 * 1024;
+}  // namespace
+
+extern "C" int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32_t absent_cta, int32_t budget_us,
+                                           void* scratch, size_t scratch_bytes, int32_t* status, float* result,
+                                           void* stream) {
+  if (!scratch || !status || !result || rounds < 1 || rounds > (1 << 20) || budget_us < 1 || budget_us > (1 << 16))
+    return fail(nullptr, AD_ERR_ARG, "ad_debug_grid_barrier_probe: bad argument");
+  if (n_ctas <= 0) n_ctas = num_sms();
+  if (absent_cta >= n_ctas) return fail(nullptr, AD_ERR_ARG, "ad_debug_grid_barrier_probe: absent_cta outside the grid");
+  if (scratch_bytes < 256 + sizeof(unsigned int) * 2 * (size_t)n_ctas || reinterpret_cast<uintptr_t>(scratch) % 256)
+    return fail(nullptr, AD_ERR_CAPACITY, "ad_debug_grid_barrier_probe: scratch too small or not 256-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaFuncSetAttribute(grid_barrier_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem) != cudaSuccess)
+    return fail(nullptr, AD_ERR_CUDA, "ad_debug_grid_barrier_probe: cudaFuncSetAttribute failed");
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, grid_barrier_probe_kernel, 256, kProbeSmem) != cudaSuccess)
+    return fail(nullptr, AD_ERR_CUDA, "ad_debug_grid_barrier_probe: occupancy query failed");
+  if (n_ctas > per_sm * num_sms()) return fail(nullptr, AD_ERR_CAPACITY, "ad_debug_grid_barrier_probe: more CTAs than the device holds at once");
+  unsigned int* ctr = static_cast<unsigned int*>(scratch);
+  unsigned int* payload = ctr + 64;
+  if (cudaMemsetAsync(scratch, 0, 256, st) != cudaSuccess || cudaMemsetAsync(result, 0, sizeof(float) * 4, st) != cudaSuccess)
+    return fail(nullptr, AD_ERR_CUDA, "ad_debug_grid_barrier_probe: memset failed");
+  unsigned long long budget_ns = (unsigned long long)budget_us * 1000ull;
+  int absent = absent_cta;
+  void* args[] = {&ctr, &payload, &rounds, &absent, &budget_ns, &status, &result};
+  // cooperative launch: the runtime refuses the launch unless all CTAs can be resident at once
+  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(grid_barrier_probe_kernel), dim3(n_ctas), dim3(256), args,
+                                              kProbeSmem, st);
+  if (e != cudaSuccess) return fail(nullptr, AD_ERR_CUDA, std::string("ad_debug_grid_barrier_probe: ") + cudaGetErrorString(e));
+  return AD_OK;
 }
 
 // ---- single-kernel entry points -----------------------------------------------------------------
@@ -1354,7 +1435,6 @@ extern "C" int ad_linear(const void* x, const void* W, const float* bias, int32_
 static __device__ __align__(256) unsigned char g_static_scratch[AD_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 void* g_static_scratch_addr[kMaxDevices] = {};
 }  // namespace
 
@@ -1375,7 +1455,11 @@ extern "C" int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dt
       return fail(nullptr, AD_ERR_CUDA, std::string("ad_vocab_argmax_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
     g_static_scratch_addr[dev] = p;
   }
-  return ad_vocab_argmax(x, emb, dtype, M, d, vocab, argmax, g_static_scratch_addr[dev], AD_STATIC_SCRATCH_BYTES, status, stream);
+  const int rc = ad_vocab_argmax(x, emb, dtype, M, d, vocab, argmax, g_static_scratch_addr[dev], AD_STATIC_SCRATCH_BYTES, status, stream);
+  if (rc != AD_OK)
+    return fail(nullptr, rc, rc == AD_ERR_ARG ? "ad_vocab_argmax_static: unsupported shape or dtype (BF16 needs d % 64 == 0 and M <= 256)"
+                                              : "ad_vocab_argmax_static: encoding a TMA descriptor or launching a kernel failed");
+  return AD_OK;
 }
 
 #ifdef AD_TRACE

@@ -12,7 +12,7 @@
 // in the epilogue: warp w reads the 32 TMEM lanes of quadrant w % 4 (tcgen05.ld 32x32b), adds the issuers' regions
 // up, and the two warps of a quadrant share its token columns.  The epilogue is a chain of dependent instructions
 // per thread, so halving each thread's share of it shortens the kernel.
-// Every mbarrier wait is bounded; on expiry the kernel latches AD_ERR_TIMEOUT, frees its TMEM and returns.
+// Every mbarrier wait is bounded in time (20 ms); on expiry the kernel latches AD_ERR_TIMEOUT, frees its TMEM and returns.
 #pragma once
 
 #include "ad_common.cuh"
@@ -26,7 +26,8 @@ constexpr int THREADS = 256;        // 8 warps: two per tensor-memory lane quadr
 constexpr int UMMA_K = 16;          // K of one tcgen05.mma kind::f16
 constexpr int A_STAGE_BYTES = BLOCK_N_FEAT * BLOCK_K * 2;   // 16 KiB
 constexpr int MAX_STAGES = 8;
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
+// Budget of a bounded wait in nanoseconds of the global timer (a legitimate wait lasts microseconds).
+constexpr unsigned long long WAIT_BUDGET_NS = 20ull * 1000 * 1000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -61,12 +62,28 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok;
 }
-// Bounded wait.  Returns false (after latching the error) when the phase did not complete in time.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i)
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: bounded by TIME, not by a poll count (one try_wait may itself suspend the thread for a while).
+// The timer is read every 64 polls.  Returns false (after latching the error) when the phase did not complete
+// within WAIT_BUDGET_NS.
+__device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, int* status, unsigned long long budget_ns) {
+  for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > budget_ns) break;
+  }
   latch_error(status, AD_ERR_TIMEOUT);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  return mbar_wait_budget(bar, parity, status, WAIT_BUDGET_NS);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {

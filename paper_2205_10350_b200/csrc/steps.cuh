@@ -47,7 +47,12 @@ enum DraftSource : int {
 struct Dims {
   int B, max_src, max_tgt, kmax;
   int bos, pad, eos, mask;
+  int vocab;
 };
+
+// Token ids that reach an embedding lookup come from the caller (source, drafts, override stream, forced tokens).
+// An id outside [0, vocab) is never used as an index: it is replaced and AD_ERR_ARG is latched.
+__device__ __forceinline__ bool id_in_vocab(int id, const Dims& dm) { return id >= 0 && id < dm.vocab; }
 
 // ---------------------------------------------------------------------------------------------
 // Suffix match of Algorithm 1, line 3, for one row, executed by one warp.
@@ -149,12 +154,14 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
       if (source == SRC_USER) dr[i] = st.user_drafts[(size_t)b * dm.kmax + i];
       if (override_stream && (source == SRC_OVERRIDE || source == SRC_KEEP))
         dr[i] = (len + i < override_len) ? override_stream[(size_t)b * override_stride + len + i] : -1;
+      // a caller-provided draft beyond the vocabulary becomes a slot that matches nothing (negative = sentinel is legal)
+      if (dr[i] >= dm.vocab) { latch_error(st.status, AD_ERR_ARG); dr[i] = -1; }
     }
     __syncwarp();
     for (int i = lane; i < k; i += 32) {
       const int m = off + i;
       int tok = (i == 0) ? st.last[b] : dr[i - 1];
-      if (tok < 0) tok = dm.pad;
+      if (tok < 0 || tok >= dm.vocab) tok = dm.pad;
       plan.tok_row[m] = b;
       plan.tok_pos[m] = len + i;
       plan.tok_id[m] = tok;
@@ -213,6 +220,12 @@ plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
   __shared__ int s_off[257];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int B = dm.B;
+  // a device-resident src_len is checked here (the host cannot see it): out-of-range lengths are clamped
+  for (int b = tid; b < B; b += 256) {
+    const int n = st.srclen[b];
+    if (n < 1 || n > dm.max_src) { latch_error(st.status, AD_ERR_ARG); st.srclen[b] = max(1, min(n, dm.max_src)); }
+  }
+  __syncthreads();
   if (tid == 0) {
     int acc = 0;
     for (int b = 0; b < B; ++b) { s_off[b] = acc; acc += st.srclen[b]; }
@@ -234,7 +247,9 @@ plan_encode_kernel(DevState st, PassPlan plan, Dims dm) {
       const int m = off + i;
       plan.tok_row[m] = b;
       plan.tok_pos[m] = i;
-      plan.tok_id[m] = st.src[(size_t)b * dm.max_src + i];
+      int id = st.src[(size_t)b * dm.max_src + i];
+      if (!id_in_vocab(id, dm)) { latch_error(st.status, AD_ERR_ARG); id = dm.pad; st.src[(size_t)b * dm.max_src + i] = id; }
+      plan.tok_id[m] = id;
       plan.kv_slot[m] = m;
       plan.att_n[m] = n;
       st.enc_slot[m] = b * dm.max_src + i;
@@ -537,7 +552,8 @@ draft_score_kernel(DevState st, PassPlan blk, Dims dm, const WT* __restrict__ em
   const int m = blockIdx.x * 8 + warp;
   if (m >= *blk.M) return;
   const int b = blk.tok_row[m];
-  const int id = st.drafts[(size_t)b * dm.kmax + (m - blk.seg_off[b])];
+  int id = st.drafts[(size_t)b * dm.kmax + (m - blk.seg_off[b])];
+  if (id >= dm.vocab) id = -1;
   float acc = 0.f;
   if (id >= 0)
     for (int i = lane; i < d; i += 32) acc = fmaf(to_f32(x[(size_t)m * d + i]), to_f32(emb[(size_t)id * d + i]), acc);
@@ -682,6 +698,7 @@ force_commit_kernel(DevState st, PassPlan blk, Dims dm, const int* tokens, const
     const int* dr = st.drafts + (size_t)b * dm.kmax;
     bool ok = n >= 0 && n <= k;
     for (int i = 0; ok && i + 1 < n; ++i) ok = tk[i] == dr[i];
+    for (int i = 0; ok && i < n; ++i) ok = id_in_vocab(tk[i], dm);      // the last one is fed to the next block
     if (!ok) { latch_error(st.status, AD_ERR_ARG); continue; }
     if (n > 0) {
       int len = st.len[b];

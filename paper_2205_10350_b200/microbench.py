@@ -4,6 +4,7 @@
   python -m paper_2205_10350_b200.microbench --op linear --M 40 --K 512 --N 2048 --reps 5
   python -m paper_2205_10350_b200.microbench --op verify --model base --batch 1 --k 16 --prefix 16 --src 32 --reps 20
   python -m paper_2205_10350_b200.microbench --op loop   --model base --sentences 4
+  python -m paper_2205_10350_b200.microbench --op gridbar
 
 Timed with CUDA events on the launching stream; prints one JSON line.
 """
@@ -40,7 +41,7 @@ def _events(stream, fn, reps, flush=None):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["vocab", "linear", "verify", "loop"])
+    ap.add_argument("--op", required=True, choices=["vocab", "linear", "verify", "loop", "gridbar"])
     ap.add_argument("--model", default="base")
     ap.add_argument("--M", type=int, default=40)
     ap.add_argument("--K", type=int, default=512)
@@ -62,7 +63,19 @@ def main():
     import ctypes as C
     out = dict(op=args.op, cold=args.cold)
 
-    if args.op in ("vocab", "linear"):
+    if args.op == "gridbar":
+        scratch = torch.zeros(8192, dtype=torch.uint8, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        result = torch.zeros(4, dtype=torch.float32, device=dev)
+        res = {}
+        for n in (0, 128, 64, 16, 2):
+            for _ in range(2):
+                assert lib.ad_debug_grid_barrier_probe(n, args.reps * 50, -1, 20000, scratch.data_ptr(), scratch.numel(),
+                                                       status.data_ptr(), result.data_ptr(), stream.cuda_stream) == 0
+                stream.synchronize()
+            res[str(n or "all")] = round(float(result[0].item()), 1)
+        out.update(ns_per_barrier_by_ctas=res, status=int(status.item()))
+    elif args.op in ("vocab", "linear"):
         M, K = args.M, args.K
         N = args.V if args.op == "vocab" else args.N
         x = torch.randn((M, K), device=dev).bfloat16()

@@ -112,15 +112,16 @@ def test_teacher_forcing_rejects_inconsistent_tokens(setup):
 
 
 def test_bounded_wait_runs_out_and_reports_timeout():
-    """A wait on a barrier that nothing completes must give up after its poll limit, latch AD_ERR_TIMEOUT and
+    """A wait on a barrier that nothing completes must give up after its time budget, latch AD_ERR_TIMEOUT and
     leave the GPU usable (no trap, no hang)."""
     import torch
     lib = binding.load()
     status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
-    polls = torch.zeros(1, dtype=torch.int32, device="cuda:0")
-    assert lib.ad_debug_wait_probe(status.data_ptr(), 64, polls.data_ptr(), None) == binding.AD_OK
+    waited = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    assert lib.ad_debug_wait_probe(status.data_ptr(), 300, waited.data_ptr(), None) == binding.AD_OK
     torch.cuda.synchronize()
-    assert int(status.item()) == binding.AD_ERR_TIMEOUT and int(polls.item()) == 64
+    assert int(status.item()) == binding.AD_ERR_TIMEOUT
+    assert 300 <= int(waited.item()) < 20000, int(waited.item())      # gave up after the budget, not after seconds
     # the context still works afterwards
     x = torch.ones((4, 64), device="cuda:0").bfloat16()
     y = binding.linear(x, x)
@@ -186,3 +187,71 @@ def test_encoders_on_two_streams_equal_encoders_in_sequence(monkeypatch):
             assert np.array_equal(x, y)
     for x, y in zip(got[0][1], got[1][1]):
         assert np.array_equal(x, y)
+
+
+def test_token_ids_and_device_side_lengths_outside_their_range_become_error_codes(setup):
+    """Ids index the embedding matrix, so every id a caller can supply is range-checked on the device before use:
+    the bad id is replaced by [PAD] (sources, fed tokens) or by a slot that matches nothing (drafts), AD_ERR_ARG is
+    reported by the next synchronising call, and only valid memory is ever read."""
+    import torch
+    dec, om = setup
+    V = dec.shape.vocab
+    good = np.array([[5, 6, 7, 8, 9, 10, 11, 12, 13, 14]], np.int32)
+    for bad_id in (V, V + 1000, -3):
+        src = good.copy()
+        src[0, 2] = bad_id
+        with pytest.raises(binding.AdError) as e:
+            dec.encode(src, [6])
+        assert e.value.code == binding.AD_ERR_ARG
+    dec.encode(good, [6])                                   # the handle is usable afterwards
+    st = om.state(good[0, :6], cap=12)
+    # a draft beyond the vocabulary: reported, and treated as a slot that matches nothing
+    drafts = np.array([[20, V, 22, 23, -1, -1]], np.int32)
+    with pytest.raises(binding.AdError) as e:
+        dec.verify_block(drafts, [4])
+    assert e.value.code == binding.AD_ERR_ARG
+    # forced tokens beyond the vocabulary are refused, the row stays where it was
+    am, n = dec.verify_block(np.array([[20, 21, 22, -1, -1, -1]], np.int32), [3])
+    with pytest.raises(binding.AdError) as e:
+        dec.force_commit(np.array([[20, 21, V + 5, -1, -1, -1]], np.int32), [3])
+    assert e.value.code == binding.AD_ERR_ARG
+    assert dec.state()[0][0] == 0
+    # device-resident source lengths cannot be seen by the host: max_src + 1 and 0 are clamped and reported
+    for bad_len in (dec.max_src + 1, 0, -4):
+        t_src = torch.tensor(good, device="cuda:0")
+        t_len = torch.tensor([bad_len], dtype=torch.int32, device="cuda:0")
+        rc = dec.lib.ad_encode(dec.h, t_src.data_ptr(), 10, t_len.data_ptr(), 1, 0)
+        assert rc == binding.AD_OK                            # asynchronous call: the check runs on the device
+        with pytest.raises(binding.AdError) as e:
+            dec.sync()
+        assert e.value.code == binding.AD_ERR_ARG
+    dec.encode(good, [6])
+    am, n = dec.verify_block(np.array([[20, 21, 22, -1, -1, -1]], np.int32), [3])
+    res = st.verify_block(0, np.array([20, 21, 22], np.int32))
+    assert np.array_equal(am[0, :3], res["pred"]) and n[0] == res["n"]
+
+
+def test_grid_barrier_passes_data_and_its_bounded_wait_runs_out():
+    """The grid-wide barrier of the persistent kernel: (a) 200 rounds over one CTA per SM, every CTA checking its
+    neighbour's word after each barrier; (b) one CTA that never arrives: the others give up after the time budget,
+    report AD_ERR_TIMEOUT and return, and the context stays usable."""
+    import torch
+    lib = binding.load()
+    scratch = torch.zeros(8192, dtype=torch.uint8, device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    result = torch.zeros(4, dtype=torch.float32, device="cuda:0")
+    rc = lib.ad_debug_grid_barrier_probe(0, 200, -1, 20000, scratch.data_ptr(), scratch.numel(), status.data_ptr(),
+                                         result.data_ptr(), None)
+    assert rc == binding.AD_OK, lib.ad_last_error(None)
+    torch.cuda.synchronize()
+    r = result.cpu().numpy()
+    assert int(status.item()) == 0 and r[1] == 200 and r[2] == 0
+    assert 100.0 < r[0] < 20000.0, r[0]                     # nanoseconds per barrier: sub-microsecond to a few microseconds
+    print(f"grid barrier over all SMs: {r[0]:.0f} ns per barrier")
+    rc = lib.ad_debug_grid_barrier_probe(0, 5, 3, 500, scratch.data_ptr(), scratch.numel(), status.data_ptr(),
+                                         result.data_ptr(), None)
+    assert rc == binding.AD_OK
+    torch.cuda.synchronize()
+    assert int(status.item()) == binding.AD_ERR_TIMEOUT and result.cpu().numpy()[1] == 0
+    x = torch.ones((4, 64), device="cuda:0").bfloat16()
+    assert float(binding.linear(x, x)[0, 0]) == 64.0
