@@ -234,6 +234,8 @@ int ad_debug_wait_probe(int32_t* status, int32_t budget_us, int32_t* waited_us, 
  * without arriving: the others' first wait then runs out after budget_us (1..65536), AD_ERR_TIMEOUT is latched in
  * *status and the kernel returns normally.  scratch: device memory, 256-byte aligned, >= 256 + 8 * n_ctas bytes.
  * result (device float[4]): [0] nanoseconds per barrier, [1] rounds completed, [2] payload mismatches (must be 0).
+ * A negative `rounds` = -(4 * rounds + v) selects a timing variant: v bit 0 = relaxed polls followed by one acquire fence instead of
+ * one acquire load per poll, v bit 1 = the barrier alone, without the payload store and check.
  * Asynchronous on `stream`.  Errors: AD_ERR_ARG, AD_ERR_CAPACITY (more CTAs than fit at once), AD_ERR_CUDA. */
 int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32_t absent_cta, int32_t budget_us, void* scratch,
                                 size_t scratch_bytes, int32_t* status, float* result, void* stream);

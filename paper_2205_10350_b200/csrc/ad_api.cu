@@ -1287,7 +1287,7 @@ namespace {
 // mismatches seen by any CTA (must be 0).
 __global__ void __launch_bounds__(256, 1)
 grid_barrier_probe_kernel(unsigned int* ctr, unsigned int* payload, int rounds, int absent, unsigned long long budget_ns,
-                          int* status, float* result) {
+                          int* status, float* result, int variant) {
   extern __shared__ uint8_t probe_smem[];    // only there to hold the SM: one CTA per SM, as in the persistent kernels
   __shared__ int flag;
   const unsigned int n = gridDim.x;
@@ -1297,14 +1297,15 @@ grid_barrier_probe_kernel(unsigned int* ctr, unsigned int* payload, int rounds, 
   if (threadIdx.x == 0) probe_smem[0] = 0;
   const unsigned long long t0 = gs::now_ns();
   for (int r = 0; r < rounds; ++r) {
+    // variant bit 0: relaxed polls + one acquire fence instead of an acquire load per poll; bit 1: no payload (barrier alone)
     unsigned int* slot = payload + (size_t)(r & 1) * n;
-    if (threadIdx.x == 0) slot[blockIdx.x] = (unsigned int)r * 4096u + blockIdx.x;
-    if (!gs::grid_barrier(ctr, gen, n, budget_ns, &flag)) {
+    if (threadIdx.x == 0 && !(variant & 2)) slot[blockIdx.x] = (unsigned int)r * 4096u + blockIdx.x;
+    if (!gs::grid_barrier(ctr, gen, n, budget_ns, &flag, (variant & 1) != 0)) {
       if (threadIdx.x == 0) latch_error(status, AD_ERR_TIMEOUT);
       break;
     }
     const unsigned int nb = (blockIdx.x + 1) % n;
-    if (threadIdx.x == 0 && __ldcg(slot + nb) != (unsigned int)r * 4096u + nb) bad++;
+    if (threadIdx.x == 0 && !(variant & 2) && __ldcg(slot + nb) != (unsigned int)r * 4096u + nb) bad++;
     ++done;
   }
   const unsigned long long t1 = gs::now_ns();
@@ -1322,6 +1323,8 @@ constexpr int kProbeSmem = 160 * 1024;
 extern "C" int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32_t absent_cta, int32_t budget_us,
                                            void* scratch, size_t scratch_bytes, int32_t* status, float* result,
                                            void* stream) {
+  int variant = 0;
+  if (rounds < 0) { variant = (-rounds) & 3; rounds = (-rounds) >> 2; }   // timing variants of the probe (see the kernel)
   if (!scratch || !status || !result || rounds < 1 || rounds > (1 << 20) || budget_us < 1 || budget_us > (1 << 16))
     return fail(nullptr, AD_ERR_ARG, "ad_debug_grid_barrier_probe: bad argument");
   if (n_ctas <= 0) n_ctas = num_sms();
@@ -1341,7 +1344,7 @@ extern "C" int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32
     return fail(nullptr, AD_ERR_CUDA, "ad_debug_grid_barrier_probe: memset failed");
   unsigned long long budget_ns = (unsigned long long)budget_us * 1000ull;
   int absent = absent_cta;
-  void* args[] = {&ctr, &payload, &rounds, &absent, &budget_ns, &status, &result};
+  void* args[] = {&ctr, &payload, &rounds, &absent, &budget_ns, &status, &result, &variant};
   // cooperative launch: the runtime refuses the launch unless all CTAs can be resident at once
   cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(grid_barrier_probe_kernel), dim3(n_ctas), dim3(256), args,
                                               kProbeSmem, st);

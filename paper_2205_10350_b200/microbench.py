@@ -68,13 +68,18 @@ def main():
         status = torch.zeros(1, dtype=torch.int32, device=dev)
         result = torch.zeros(4, dtype=torch.float32, device=dev)
         res = {}
-        for n in (0, 128, 64, 16, 2):
-            for _ in range(2):
-                assert lib.ad_debug_grid_barrier_probe(n, args.reps * 50, -1, 20000, scratch.data_ptr(), scratch.numel(),
-                                                       status.data_ptr(), result.data_ptr(), stream.cuda_stream) == 0
-                stream.synchronize()
-            res[str(n or "all")] = round(float(result[0].item()), 1)
-        out.update(ns_per_barrier_by_ctas=res, status=int(status.item()))
+        rounds = args.reps * 50
+        # variants (negative rounds = -(rounds * 4 + v)): v bit 0 = relaxed polls + one fence, bit 1 = barrier without payload
+        names = {0: "acquire_polls_with_payload", 1: "relaxed_polls_with_payload", 2: "acquire_polls_barrier_only", 3: "relaxed_polls_barrier_only"}
+        for v, name in names.items():
+            res[name] = {}
+            for n in (0, 128, 64, 16, 2):
+                for _ in range(2):
+                    assert lib.ad_debug_grid_barrier_probe(n, -(rounds * 4 + v), -1, 20000, scratch.data_ptr(), scratch.numel(),
+                                                           status.data_ptr(), result.data_ptr(), stream.cuda_stream) == 0
+                    stream.synchronize()
+                res[name][str(n or "all")] = round(float(result[0].item()), 1)
+        out.update(ns_per_barrier_by_variant_and_ctas=res, status=int(status.item()))
     elif args.op in ("vocab", "linear"):
         M, K = args.M, args.K
         N = args.V if args.op == "vocab" else args.N
