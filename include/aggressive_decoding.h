@@ -220,6 +220,14 @@ int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_
 /* Debug: FP32 copy of the verifier's encoder memory of row b, [src_len_b, d_model] (device pointer). */
 int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size_t capacity_elems);
 
+/* Debug: stage timeline of the last persistent decoder pass (the single-kernel form of the decoder stack that handles
+ * BF16 models with 64-wide heads and passes of at most 64 packed tokens).  With AD_MEGA_TIMELINE=1 in the environment
+ * when the handle is created, CTA 0 of that kernel stamps the GPU's global nanosecond timer twice per stage: when the
+ * stage's inputs have become visible, and after it has signalled its own part done.  stamps (host, >= 2 * n_stages
+ * entries) receives them in stage order: per decoder layer QKV, self-attention, Wo, cross-Q, cross-attention, cross-Wo,
+ * FFN1, FFN2; then the vocabulary projection.  Synchronises the stream. */
+int ad_debug_stage_timeline(ad_handle* h, uint64_t* stamps, int32_t capacity, int32_t* n_stages);
+
 /* Debug: exercises the bounded-wait mechanism that every mbarrier wait of the GEMM kernels uses (a wait gives up
  * after a time budget measured on the GPU's global timer: 20 ms in the kernels, budget_us here).  Launches one tiny
  * kernel that waits, for at most budget_us (1..65536) microseconds, on a barrier phase that nothing completes; the

@@ -21,7 +21,7 @@ AD_MODE_IAD, AD_MODE_GAD = 0, 1
 EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
     "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync", "ad_set_acceptance",
-    "ad_debug_logits", "ad_debug_encoder_memory", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
+    "ad_debug_logits", "ad_debug_encoder_memory", "ad_debug_stage_timeline", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
     "ad_vocab_argmax_static", "ad_debug_wait_probe", "ad_debug_grid_barrier_probe",
     "ad_linear",
 ]
@@ -89,6 +89,7 @@ def load():
         "ad_set_acceptance": (C.c_int, [vp, C.c_int32, C.c_float]),
         "ad_debug_logits": (C.c_int, [vp, i32, vp, sz]),
         "ad_debug_encoder_memory": (C.c_int, [vp, i32, vp, sz]),
+        "ad_debug_stage_timeline": (C.c_int, [vp, vp, i32, vp]),
         "ad_vocab_argmax_scratch_bytes": (sz, [i32, i32]),
         "ad_vocab_argmax": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, sz, vp, vp]),
         "ad_vocab_argmax_static": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
@@ -248,6 +249,13 @@ class AggressiveDecoder:
         self._check(self.lib.ad_debug_logits(self.h, which, C.c_void_p(t.data_ptr()), t.numel()), self.h)
         self.sync()
         return t.cpu().numpy()
+
+    def debug_stage_timeline(self):
+        """Per-stage (inputs visible, signalled) global-timer stamps of the last persistent decoder pass, in ns."""
+        buf = np.zeros(2 * (8 * self.shape.n_dec + 1), np.uint64)
+        n = C.c_int32()
+        self._check(self.lib.ad_debug_stage_timeline(self.h, buf.ctypes.data, buf.size, C.byref(n)), self.h)
+        return buf.reshape(-1, 2)
 
     def debug_encoder_memory(self, b, src_len):
         t = self.torch.empty((src_len, self.shape.d_model), dtype=self.torch.float32, device=self.dev)

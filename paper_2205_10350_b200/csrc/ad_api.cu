@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "grid_sync.cuh"
+#include "mega.cuh"
 #include "steps.cuh"
 
 using namespace ad;
@@ -130,6 +131,19 @@ struct ad_handle {
   std::map<std::string, GraphEntry> graphs;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
   int launches = 0;          // kernels launched by the last ad_generate (direct) or per graph replay
+  // Persistent decoder pass (one kernel for the decoder stack + projection): per pass kind, whether it applies and its
+  // fixed arguments; device-resident tables of tensor maps (per model) and of per-layer pointers (per pass kind).
+  struct MegaPass { bool on = false; mega::Params p; };
+  MegaPass mega[PK_COUNT];
+  int mega_cs = 0, mega_nc = 0;
+  size_t mega_smem = 0;
+  CUtensorMap* mega_maps[2] = {nullptr, nullptr};          // [0] verifier, [1] drafter
+  mega::LayerPtrs* mega_layers[2] = {nullptr, nullptr};    // [0] verification pass, [1] drafter pass
+  float* mega_stats[2] = {nullptr, nullptr};
+  unsigned long long* mega_timeline = nullptr;
+#ifdef AD_MEGA_DEBUG
+  float* mega_dbg = nullptr;
+#endif
   unsigned long long cond_handle = 0;   // non-zero only while the body of a device-side `while` node is captured
 };
 
@@ -284,6 +298,15 @@ size_t layout(ad_handle* h, void* base) {
   h->max_pos = std::max(c.max_src, c.max_tgt + 1);
   h->pe = (float*)bp.take(sizeof(float) * (size_t)h->max_pos * d);
   h->ovr = (int*)bp.take(sizeof(int) * (size_t)B * c.max_tgt);
+  for (int i = 0; i < 2; ++i) {
+    h->mega_maps[i] = (CUtensorMap*)bp.take(sizeof(CUtensorMap) * (size_t)(6 * c.n_dec + 1));
+    h->mega_layers[i] = (mega::LayerPtrs*)bp.take(sizeof(mega::LayerPtrs) * (size_t)c.n_dec);
+    h->mega_stats[i] = (float*)bp.take(sizeof(float) * 2 * (size_t)(d / 128 + 1) * M_all);
+  }
+  h->mega_timeline = (unsigned long long*)bp.take(sizeof(unsigned long long) * 2 * (size_t)(mega::ST_PER_LAYER * c.n_dec + 1));
+#ifdef AD_MEGA_DEBUG
+  h->mega_dbg = (float*)bp.take(sizeof(float) * 16 * 32 * 4);
+#endif
   for (int k = 0; k < PK_COUNT; ++k) plan_take(bp, h->pass[k].plan, B, h->pass[k].M_cap);
   DevState& s = h->st;
   auto ints = [&](size_t n) { return (int*)bp.take(sizeof(int) * n, 256); };
@@ -293,6 +316,7 @@ size_t layout(ad_handle* h, void* base) {
   s.drafts = ints((size_t)B * c.kmax); s.pred = ints((size_t)B * c.kmax); s.n_acc = ints(B);
   s.stat_it = ints(B); s.stat_acc = ints(B); s.stat_off = ints(B);
   s.loop_it = ints(4); s.status = ints(4); s.all_fin = ints(4);
+  s.sync_ctr = (unsigned int*)ints((size_t)mega::SYNC_COUNTERS * mega::SYNC_STRIDE);
   s.cross_base = ints(B);
   s.gidx = ints((size_t)B * c.kmax);
   s.enc_slot = ints((size_t)B * c.max_src);
@@ -363,6 +387,7 @@ bool g_use_graph_encode = true;   // AD_NO_ENCODE_GRAPH=1: launch the encoder ke
 bool g_two_stream_encode = true;   // AD_NO_CONCURRENT_ENCODERS=1: the drafter's encoder after the verifier's, on one stream
 bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
 bool g_fuse_attn_proj = true;   // AD_NO_ATTN_PROJ=1: attention and its output projection always as separate kernels
+bool g_use_mega = true;         // AD_NO_MEGA=1: never use the persistent decoder-pass kernel (always the kernel chain)
 
 // Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
 // themselves wait with griddepcontrol.wait before touching anything a predecessor writes).
@@ -602,6 +627,142 @@ int ffn_sublayer(ad_handle* h, int pk, const Mat& w1, const float* b1, const Mat
   return layernorm(h, pc, ns, b2, lng, lnb);
 }
 
+
+// ---- persistent decoder pass ---------------------------------------------------------------------------------
+
+// Cluster size for the K split of the projections: the K blocks of d_model and of d_ffn must divide evenly, and a CTA's
+// share of the B operand (its K blocks x 64 tokens x 128 bytes) must fit the 64 KB operand area.
+int mega_cluster_size(const ad_model_cfg& c) {
+  for (int cs : {8, 4}) {
+    const int kd = c.d_model / 64, kf = c.d_ffn / 64;
+    if (kd % cs || kf % cs) continue;
+    if ((kf / cs) * mega::NT_MAX * 128 > 64 * 1024) continue;
+    return cs;
+  }
+  return 0;
+}
+
+// Fills the device tables and the fixed kernel arguments of the persistent decoder pass; leaves mega[pk].on false for
+// pass kinds (or models, or devices) it does not apply to.  Runs once, from ad_create.
+int mega_setup(ad_handle* h) {
+  const ad_model_cfg& c = h->cfg;
+  if (!g_use_mega || !h->bf16 || c.d_model / c.n_heads != 64 || c.d_model % 128 || c.d_ffn % 128) return AD_OK;
+  if (mega::ST_PER_LAYER * c.n_dec + 1 > mega::SYNC_COUNTERS) return AD_OK;
+  const int cs = mega_cluster_size(c);
+  if (!cs) return AD_OK;
+  // shared memory: alignment slack + weight ring + work area (see the kernel), sized for the larger of the two passes
+  int max_optin = 0, dev = current_device();
+  cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  int cap = 0;
+  for (int pk : {PK_VERIFY, PK_DRAFT})
+    if (h->pass[pk].M_cap <= mega::NT_MAX && (pk == PK_VERIFY || c.has_drafter)) cap = std::max(cap, h->pass[pk].M_cap);
+  if (cap == 0) return AD_OK;
+  const int ntcap = (cap + 15) / 16 * 16;
+  const int b_bytes = (std::max(c.d_model, c.d_ffn) / 64 / cs) * ntcap * 128;
+  const int red_bytes = ntcap * mega::RED_LD * 4;
+  const int work = std::max(std::max(b_bytes + 2 * red_bytes, (c.d_model / 64) * ntcap * 128), mega::ATT_SMEM);
+  int ring = (max_optin - 1024 - work - 4096) / mega::TILE_A;     // 4096: the kernel's static control block
+  if (ring > mega::MAX_RING) ring = mega::MAX_RING;
+  if (ring < 4) return AD_OK;
+  const size_t smem = 1024 + (size_t)ring * mega::TILE_A + (size_t)work;
+  if (cudaFuncSetAttribute(mega::decoder_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return AD_OK;
+  }
+  // how many clusters the device holds at once
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(cs * 64); cfg.blockDim = dim3(mega::THREADS); cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n_clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&n_clusters, mega::decoder_pass_kernel, &cfg) != cudaSuccess || n_clusters < 2) {
+    cudaGetLastError();
+    return AD_OK;
+  }
+  h->mega_cs = cs; h->mega_nc = n_clusters; h->mega_smem = smem;
+
+  const int d = c.d_model, L = c.n_dec;
+  const size_t self_layer = (size_t)c.max_tgt * c.max_batch * d * h->esz;
+  const size_t cross_layer = (size_t)c.max_src * c.max_batch * d * h->esz;
+  for (int which = 0; which < 2; ++which) {          // 0: verification pass (verifier), 1: drafter pass (drafter)
+    Model& m = which == 0 ? h->ar : h->nar;
+    if (!m.present) continue;
+    const int pk = which == 0 ? PK_VERIFY : PK_DRAFT;
+    if (h->pass[pk].M_cap > mega::NT_MAX) continue;
+    std::vector<CUtensorMap> maps((size_t)6 * L + 1);
+    std::vector<mega::LayerPtrs> lp((size_t)L);
+    for (int l = 0; l < L; ++l) {
+      DecLayer& D = m.dec[l];
+      const Mat* mats[6] = {&D.wqkv, &D.wo, &D.cq, &D.co, &D.w1, &D.w2};
+      for (int i = 0; i < 6; ++i) maps[(size_t)6 * l + i] = mats[i]->map;
+      mega::LayerPtrs& P = lp[l];
+      P.bqkv = D.bqkv; P.bo = D.bo; P.ln1g = D.ln1g; P.ln1b = D.ln1b; P.cbq = D.cbq; P.cbo = D.cbo; P.ln2g = D.ln2g; P.ln2b = D.ln2b;
+      P.b1 = D.b1; P.b2 = D.b2; P.ln3g = D.ln3g; P.ln3b = D.ln3b;
+      P.kself = (bf16*)(which == 0 ? (char*)h->kself + l * self_layer : (char*)h->ktmp);
+      P.vself = (bf16*)(which == 0 ? (char*)h->vself + l * self_layer : (char*)h->vtmp);
+      P.kenc = (const bf16*)((char*)m.kenc + l * cross_layer);
+      P.venc = (const bf16*)((char*)m.venc + l * cross_layer);
+    }
+    maps[(size_t)6 * L] = m.emb.map;
+    AD_CUDA(h, cudaMemcpyAsync(h->mega_maps[which], maps.data(), sizeof(CUtensorMap) * maps.size(), cudaMemcpyHostToDevice, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(h->mega_layers[which], lp.data(), sizeof(mega::LayerPtrs) * lp.size(), cudaMemcpyHostToDevice, h->stream));
+    AD_CUDA(h, cudaStreamSynchronize(h->stream));     // the host vectors go out of scope
+    mega::Params& p = h->mega[pk].p;
+    p = mega::Params{};
+    p.d = d; p.H = c.n_heads; p.F = c.d_ffn; p.V = c.vocab; p.L = L;
+    p.qchunks = (h->pass[pk].seg_max + 7) / 8;
+    p.maps = h->mega_maps[which]; p.layers = h->mega_layers[which];
+    p.plan = h->pass[pk].plan;
+    p.cross_base = h->st.cross_base; p.srclen = h->st.srclen;
+    p.emb = (const bf16*)m.emb.ptr; p.pe = h->pe;
+    p.emb_scale = sqrtf((float)d); p.eps = c.ln_eps; p.att_scale = 1.0f / sqrtf(64.f);
+    p.x[0] = h->y; p.x[1] = h->pre;
+    p.stats[0] = h->mega_stats[0]; p.stats[1] = h->mega_stats[1];
+    p.M_cap = h->pass[pk].M_cap;
+    p.q = (bf16*)h->qbuf; p.attn = (bf16*)h->abuf.ptr; p.hid = (bf16*)h->hbuf.ptr;
+    p.yb_out = (bf16*)(which == 0 ? h->yb.ptr : h->xg.ptr);
+    p.vocab_M = which == 0 ? nullptr : h->pass[PK_VERIFY].plan.M;
+    p.vocab_rows = which == 0 ? nullptr : h->st.gidx;
+    p.part_val = h->part_val; p.part_idx = h->part_idx; p.n_vtiles = h->n_vtiles;
+    p.sync_ctr = h->st.sync_ctr; p.status = h->st.status;
+    p.ring = ring; p.b_bytes = b_bytes; p.red_bytes = red_bytes;
+    p.timeline = nullptr;
+    h->mega[pk].on = true;
+  }
+  return AD_OK;
+}
+
+bool mega_applies(const ad_handle* h, int pk) {
+  return h->mega[pk].on && !(pk == PK_VERIFY && h->beta >= 1);
+}
+
+// One launch: decoder stack of pass pk and the projection's per-tile arg-max partials.
+int mega_launch(ad_handle* h, int pk) {
+  mega::Params p = h->mega[pk].p;
+  p.B = h->dims.B;
+  static const bool trace = [] { const char* e = getenv("AD_MEGA_TIMELINE"); return e && e[0] == '1'; }();
+  p.timeline = trace ? h->mega_timeline : nullptr;
+#ifdef AD_MEGA_DEBUG
+  { const char* e = getenv("AD_MEGA_STOP"); p.debug_stop = e ? atoi(e) : 1 << 20; }
+  p.dbg = h->mega_dbg;
+#endif
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(h->mega_cs * h->mega_nc); cfg.blockDim = dim3(mega::THREADS);
+  cfg.dynamicSmemBytes = h->mega_smem; cfg.stream = h->stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = h->mega_cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 2 : 1;
+  h->launches++;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, mega::decoder_pass_kernel, p);
+  if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("persistent decoder pass launch: ") + cudaGetErrorString(e));
+  return AD_OK;
+}
+
 // Decoder stack over the packed tokens of pass pk (verification: cached, block-causal; drafter: no cache,
 // unmasked).  Leaves the final hidden states in yb.
 int decoder_pass(ad_handle* h, int pk, Model& m) {
@@ -676,7 +837,7 @@ void swap_side(ad_handle* h) {
 
 // Output projection fused with arg-max over X (yb for the verifier, the gathered mask rows for the drafter),
 // then the final reduction and (verifier) the draft compare.
-int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto_commit) {
+int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto_commit, bool partials_ready = false) {
   PassCfg& pc = h->pass[PK_VERIFY];
   GemmParams p = {};
   p.part_val = h->part_val; p.part_idx = h->part_idx;
@@ -689,7 +850,7 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
     else AD_CUDA(h, launch_k(draft_score_kernel<float, float>, sgrid, dim3(256), 0, h->stream, h->st, pc.plan, h->dims, (const float*)m.emb.ptr, (const float*)X.ptr, d, h->draft_val, h->draft_id));
     p.draft_val = h->draft_val; p.draft_id = h->draft_id; p.part_cnt = h->part_cnt;
   }
-  AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
+  if (!partials_ready) AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   h->launches++;
   AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
                       pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
@@ -711,6 +872,10 @@ int draft_stage(ad_handle* h, int k_cap) {
   AD_TRY(prepare_verify(h, SRC_SIZES, k_cap, nullptr, 0));
   h->launches++;
   AD_CUDA(h, launch_k(plan_draft_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->pass[PK_DRAFT].plan, h->dims));
+  if (mega_applies(h, PK_DRAFT)) {      // decoder stack, gather of the mask rows and projection in one kernel
+    AD_TRY(mega_launch(h, PK_DRAFT));
+    return vocab_stage(h, h->nar, h->xg, 1, 0, true);
+  }
   AD_TRY(decoder_pass(h, PK_DRAFT, h->nar));
   const int d = h->cfg.d_model;
   PassCfg& pv = h->pass[PK_VERIFY];
@@ -721,6 +886,10 @@ int draft_stage(ad_handle* h, int k_cap) {
 }
 
 int verify_stage(ad_handle* h, int auto_commit) {
+  if (mega_applies(h, PK_VERIFY)) {
+    AD_TRY(mega_launch(h, PK_VERIFY));
+    return vocab_stage(h, h->ar, h->yb, 0, auto_commit, true);
+  }
   AD_TRY(decoder_pass(h, PK_VERIFY, h->ar));
   return vocab_stage(h, h->ar, h->yb, 0, auto_commit);
 }
@@ -809,6 +978,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   { const char* e = getenv("AD_NO_ENCODE_GRAPH"); g_use_graph_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_CONCURRENT_ENCODERS"); g_two_stream_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ATTN_PROJ"); g_fuse_attn_proj = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_NO_MEGA"); g_use_mega = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();
@@ -862,6 +1032,10 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
     mp->ckv_all.ptr = mp->ckv_pack; mp->ckv_all.N = cfg->n_dec * 2 * d; mp->ckv_all.K = d;
     if (h->bf16) okc = okc && make_map(&mp->ckv_all.map, mp->ckv_pack, mp->ckv_all.N, d, tc::BLOCK_N_FEAT);
     if (!okc) return bail(AD_ERR_CUDA, "gathering the cross-attention key/value projections failed");
+  }
+  {
+    const int rcm = mega_setup(h);
+    if (rcm != AD_OK) return bail(rcm, h->err);
   }
   // Sinusoidal positional table PE(p, 2i) = sin(p / 10000^(2i/d)), PE(p, 2i+1) = cos(.), evaluated in double.
   {
@@ -1253,6 +1427,41 @@ extern "C" int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size
   if (h->bf16) to_f32_kernel<bf16><<<64, 256, 0, h->stream>>>((const bf16*)h->encmem + start, mem, n);
   else to_f32_kernel<float><<<64, 256, 0, h->stream>>>((const float*)h->encmem + start, mem, n);
   AD_CUDA(h, cudaGetLastError());
+  return AD_OK;
+}
+
+#ifdef AD_MEGA_DEBUG
+// Debugging builds only: raw copy of an internal buffer (0/1: x, 2/3: statistics, 4: q, 5: attention output, 6: FFN hidden,
+// 7: yb, 8/9: self-attention keys / values of layer `layer`).
+extern "C" int ad_debug_peek(ad_handle* h, int which, int layer, void* dst, size_t bytes) {
+  const size_t self_layer = (size_t)h->cfg.max_tgt * h->cfg.max_batch * h->cfg.d_model * h->esz;
+  const void* src = nullptr;
+  switch (which) {
+    case 0: src = h->y; break;
+    case 1: src = h->pre; break;
+    case 2: src = h->mega_stats[0]; break;
+    case 3: src = h->mega_stats[1]; break;
+    case 4: src = h->qbuf; break;
+    case 5: src = h->abuf.ptr; break;
+    case 6: src = h->hbuf.ptr; break;
+    case 7: src = h->yb.ptr; break;
+    case 8: src = (char*)h->kself + layer * self_layer; break;
+    case 9: src = (char*)h->vself + layer * self_layer; break;
+    case 12: src = h->mega_dbg; break;
+    default: return AD_ERR_ARG;
+  }
+  cudaStreamSynchronize(h->stream);
+  return cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? AD_OK : AD_ERR_CUDA;
+}
+#endif
+
+extern "C" int ad_debug_stage_timeline(ad_handle* h, uint64_t* stamps, int32_t capacity, int32_t* n_stages) {
+  if (!h || !stamps || !n_stages) return AD_ERR_ARG;
+  const int n = mega::ST_PER_LAYER * h->cfg.n_dec + 1;
+  if (capacity < 2 * n) return fail(h, AD_ERR_CAPACITY, "timeline buffer too small");
+  AD_CUDA(h, cudaStreamSynchronize(h->stream));
+  AD_CUDA(h, cudaMemcpy(stamps, h->mega_timeline, sizeof(uint64_t) * 2 * (size_t)n, cudaMemcpyDeviceToHost));
+  *n_stages = n;
   return AD_OK;
 }
 

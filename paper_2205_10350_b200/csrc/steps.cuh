@@ -34,6 +34,8 @@ struct DevState {
   int* user_k;     // [B] staging of caller-provided k / n
   int* user_n;     // [B]
   int* user_drafts;// [B, kmax]
+  unsigned int* sync_ctr;  // [128 x 32] per-stage arrival counters of the persistent decoder pass (one per 128-byte line);
+                           // every planning kernel that precedes such a pass clears them
 };
 
 enum DraftSource : int {
@@ -140,6 +142,7 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
     *plan.M = acc;
     st.loop_it[1] = 0;   // rows-done counter of the accept kernel: every iteration starts from zero
   }
+  if (tid < 128) st.sync_ctr[tid * 32] = 0u;
   __syncthreads();
   for (int b = warp; b < B; b += 8) {
     const int k = s_k[b], off = s_off[b], len = st.len[b];
@@ -192,6 +195,7 @@ plan_draft_kernel(DevState st, PassPlan blk, PassPlan plan, Dims dm) {
     s_off[B] = acc;
     *plan.M = acc;
   }
+  if (tid < 128) st.sync_ctr[tid * 32] = 0u;
   __syncthreads();
   for (int b = warp; b < B; b += 8) {
     const int k = blk.seg_len[b], len = st.len[b], off = s_off[b];
