@@ -11,6 +11,12 @@ value = verified (accepted) tokens per second over the whole job.
 N > 1 (launched with torch.distributed.run): every rank decodes its own 64 sentences (replicas, no
 collective on the data path); the timed region is bracketed by barriers and the reported time is the
 maximum over ranks.
+
+The JSON line's `roofline` is the verification step (the unit of the path): algorithmic bytes of one loop
+iteration divided by its device time inside the decode loop, against the measured HBM peak.  Beside it:
+`kernels` (every kernel of one step timed on its own), `tensor_regime` (batch 32 x block 64 against the BF16
+tensor peak), `step_points` (fixed-shape verification steps, L2-warm and L2-flushed), `workloads` (the batched,
+drafter-based and long-source recipes with the CPU checker's bounded sample beside each).
 """
 from __future__ import annotations
 
@@ -36,9 +42,6 @@ WL = synth.WORKLOADS[2]
 N_SENT = WL.n_batches
 KMAX = 40                      # outputs are at most 40 tokens, so the block cap of 64 never binds
 METRIC, UNIT = "verified_tokens_per_s", "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the projection kernel at this exact shape
-# (profiles/vocab_argmax_gemm_base_M40_ncu_full.txt); set to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES = 32855040   # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/vocab_argmax_gemm_base_M40_ncu_full.txt)
 WORKLOAD_DESC = ("transformer-base (6+6, d512, h8, ffn2048, vocab 32000, bf16) GEC-shaped input-guided decoding, batch 1, "
                  "source length U[12,40], drafts = own greedy output with 10% of tokens replaced, block = remaining "
                  "length (cap 64 never binds)")
@@ -48,8 +51,9 @@ def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
 def sentence_inputs(rank):
@@ -71,6 +75,23 @@ def reduce_max_sum(dist, dev, seconds_or_ms, count):
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return float(t.item()), int(n.item())
+
+
+def weight_bytes(shape):
+    """Algorithmic weight bytes of one verification step: decoder layers (cross-attention K/V projections excluded:
+    they run once per sentence in the encoder pass) + the output projection."""
+    d, F, V, L = shape.d_model, shape.d_ffn, shape.vocab, shape.n_dec
+    s = 2 if shape.dtype == "bf16" else 4
+    return (L * (6 * d * d + 2 * d * F) + V * d) * s
+
+
+def step_bytes(shape, sum_src, sum_keys, sum_k, n_steps=1):
+    """Algorithmic bytes of n_steps verification steps: weights per step, cross-attention K/V of every active row
+    (sum_src source tokens), self-attention K/V read (sum_keys = sum of len + k) and written (sum_k block tokens)."""
+    d, L = shape.d_model, shape.n_dec
+    s = 2 if shape.dtype == "bf16" else 4
+    per_tok = 2 * L * d * s
+    return n_steps * weight_bytes(shape) + per_tok * (sum_src + sum_keys + sum_k)
 
 
 class ClockSampler:
@@ -112,9 +133,11 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------------
+# CPU checker arms (the checker as it stands, on the machine's host cores, bounded samples)
+# ------------------------------------------------------------------------------------------------------
 def oracle_sample(seconds, rank=0):
-    """The CPU checker as it stands, on a bounded sample of the same workload: whole sentences (encode +
-    draft-verify loop on the checker's own corrupted greedy stream) until `seconds` have passed."""
+    """Headline workload: whole sentences (encode + draft-verify loop on the checker's own corrupted greedy stream)
+    until `seconds` have passed."""
     from oracle import ad_oracle as O
     w = synth.make_weights(synth.BASE, 0)
     om = O.Model(synth.BASE, w, max_pos=64)
@@ -134,7 +157,41 @@ def oracle_sample(seconds, rank=0):
             break
     return dict(value=tokens / t_total, unit=UNIT, cores=O.threads(), kind="oracle",
                 sample=f"first {n_sent} of {N_SENT} sentences of the workload ({tokens} tokens, {iters} verify iterations, "
-                       f"{t_total:.1f} s), encoder included"), t_total, tokens, n_sent
+                       f"{t_total:.1f} s), encoder included",
+                ms_per_verify_step=1e3 * t_total / max(1, iters)), t_total, tokens, n_sent
+
+
+def oracle_workload_sample(index, seconds, weights, nar_weights=None):
+    """Bounded sample of one of the other workload recipes on the CPU checker: rows of its first batch, one after the
+    other (encode + draft-verify loop; with a drafter model its forward runs every iteration and its block is then
+    replaced by the corrupted stream, as on the GPU), until `seconds` have passed."""
+    from oracle import ad_oracle as O
+    wl = synth.WORKLOADS[index]
+    src, lens = synth.make_sources(wl, 0)
+    max_len = synth.max_out_lens(wl, lens)
+    cap = int(max(max_len))
+    om = O.Model(wl.shape, weights, max_pos=max(wl.src_len_hi, cap) + 2)
+    on = O.Model(wl.shape, nar_weights, max_pos=max(wl.src_len_hi, cap) + 2) if nar_weights is not None else None
+    tokens, t_total, rows, iters = 0, 0.0, 0, 0
+    for b in range(wl.batch):
+        st0 = om.state(src[b, : lens[b]])
+        g, _ = st0.greedy(int(max_len[b]))
+        gg = np.full((1, cap), synth.PAD, np.int32); gg[0, : len(g)] = g
+        stream = synth.corrupt_stream(gg, [len(g)], wl.agreement, wl.shape.vocab, wl.index, b)[0]
+        t0 = time.perf_counter()
+        st = om.state(src[b, : lens[b]])
+        if on is not None:
+            out, tr = st.gad(on, wl.k, int(max_len[b]), override=stream)
+        else:
+            out, tr = st.draft_verify_stream(stream, min(wl.k, cap), int(max_len[b]))
+        t_total += time.perf_counter() - t0
+        tokens += len(out); rows += 1; iters += tr["iterations"]
+        if t_total >= seconds:
+            break
+    return dict(value=tokens / t_total, unit=UNIT, cores=O.threads(), kind="oracle",
+                ms_per_iteration=1e3 * t_total / max(1, iters),
+                sample=f"{rows} of {wl.batch} rows of the first batch, one at a time ({tokens} tokens, {iters} iterations, "
+                       f"{t_total:.1f} s), encoder(s) and drafter included")
 
 
 def run_reference(args, rank, world):
@@ -158,6 +215,129 @@ def run_reference(args, rank, world):
 
 
 # ------------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------------
+def _events(stream, fn, reps, flush=None, warm=3):
+    """Device time of fn per call in microseconds: everything is enqueued, then the stream is synchronised once."""
+    import torch
+    evs = []
+    with torch.cuda.stream(stream):
+        for i in range(reps + warm):
+            if flush is not None:
+                flush.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            evs.append((a, b))
+    stream.synchronize()
+    return [a.elapsed_time(b) * 1e3 for a, b in evs[warm:]]
+
+
+def kernel_table(dec, shape, drafts, k, pk):
+    """Every kernel of one verification step timed on its own (an event in front of every launch, programmatic
+    dependent launch off), grouped by what was launched; bytes = algorithmic bytes of that kernel's launches."""
+    dec.profile_verify(drafts, [k])                        # warm
+    runs = [dec.profile_verify(drafts, [k]) for _ in range(5)]
+    n = len(runs[0])
+    med = [statistics.median(r[i][1] for r in runs) for i in range(n)]
+    d, F = shape.d_model, shape.d_ffn
+    groups = {}
+    for (name, _), us in zip(runs[0], med):
+        g = groups.setdefault(name, dict(name=name, launches=0, us=0.0, bytes=0))
+        g["launches"] += 1; g["us"] += us
+        if name.startswith("gemm_"):
+            N, K = (int(t[1:]) for t in name.split()[1:3])
+            out_b = 4 if "f32" in name else (0 if "argmax" in name else 2)
+            g["bytes"] += N * K * 2 + k * K * 2 + k * N * out_b
+        elif name.startswith("attention"):
+            g["bytes"] += 2 * 40 * d * 2 + 2 * k * d * 2 + (d * d * 2 + 8 * k * d * 4 if "out_proj" in name else 0)
+        elif "layernorm" in name:
+            g["bytes"] += 9 * k * d * 4 + k * d * 6
+    total = sum(g["us"] for g in groups.values())
+    rows = []
+    for g in sorted(groups.values(), key=lambda g: -g["us"]):
+        rows.append(dict(name=g["name"], launches=g["launches"], us_total=round(g["us"], 2), share=round(g["us"] / total, 4),
+                         algorithmic_bytes=g["bytes"] or None,
+                         frac_of_hbm_peak=round(g["bytes"] / (g["us"] * 1e-6) / 1e9 / pk["hbm_gbs"], 4) if g["bytes"] else None))
+    return dict(shape=f"block of {k} tokens on an empty prefix, source {dec.max_src}", launches=n, us_serialised=round(total, 1),
+                note="each kernel bracketed by its own pair of events, launches serialised (no programmatic dependent "
+                     "launch): sum exceeds the in-loop step time; shares are what to read", kernels=rows)
+
+
+def fixed_step(binding, shape, w, pk, B, k, prefix, S, reps=30, flush=None):
+    """Verification steps of one fixed shape (direct launches, verify + discard so that every repetition sees the same
+    prefix).  Returns (microseconds L2-warm, microseconds with L2 flushed before every step or None)."""
+    import torch
+    dec = binding.AggressiveDecoder(shape, w, max_batch=B, max_src=S, max_tgt=max(prefix + k, 8), kmax=k)
+    r = np.random.default_rng(0)
+    dec.encode(r.integers(4, shape.vocab, size=(B, S)).astype(np.int32), np.full(B, S, np.int32))
+    left = prefix
+    while left > 0:
+        n = min(left, k)
+        toks = r.integers(4, shape.vocab, size=(B, k)).astype(np.int32)
+        dec.verify_block(toks, np.full(B, n, np.int32)); dec.force_commit(toks, np.full(B, n, np.int32))
+        left -= n
+    dev = dec.dev
+    d_t = torch.tensor(r.integers(4, shape.vocab, size=(B, k)).astype(np.int32), device=dev)
+    k_t = torch.full((B,), k, dtype=torch.int32, device=dev)
+    a_t = torch.zeros((B, k), dtype=torch.int32, device=dev); n_t = torch.zeros(B, dtype=torch.int32, device=dev)
+    z_t = torch.zeros(B, dtype=torch.int32, device=dev)
+
+    def fn():
+        dec.verify_block_device(d_t, k_t, a_t, n_t)
+        dec.commit_device(z_t)
+    warm = statistics.mean(_events(dec.stream, fn, reps))
+    cold = statistics.mean(_events(dec.stream, fn, max(5, reps // 3), flush)) if flush is not None else None
+    dec.sync(); dec.close()
+    return warm, cold
+
+
+def run_workload(binding, index, w, wn, dev, n_batches, oracle_seconds, pk):
+    """One of the other workload recipes through ad_generate (device-resident inputs): batched input-guided decoding,
+    or drafter-based decoding with the drafter forward timed and its block then replaced by the corrupted stream."""
+    import torch
+    wl = synth.WORKLOADS[index]
+    gad = wl.mode == "GAD"
+    cap = wl.max_out if wl.max_out > 0 else wl.src_len_hi
+    dec = binding.AggressiveDecoder(wl.shape, w, wn if gad else None, max_batch=wl.batch, max_src=wl.src_len_hi, max_tgt=cap,
+                                    kmax=min(wl.k, cap), device=str(dev))
+    k = min(wl.k, cap)
+    tot = dict(accepted=0, iterations=0, row_iterations=0, offered=0, device_ms=0.0, encode_ms=0.0, wall_ms=0.0)
+    sum_src = 0
+    for bi in range(n_batches):
+        src, lens = synth.make_sources(wl, bi)
+        max_len = synth.max_out_lens(wl, lens)
+        g_out, _ = dec.generate(src, lens, mode="IAD", k=1, max_len=max_len)      # own greedy output (untimed)
+        g = np.full((wl.batch, cap), synth.PAD, np.int32); gl = np.zeros(wl.batch, np.int32)
+        for b in range(wl.batch):
+            g[b, : len(g_out[b])] = g_out[b]; gl[b] = len(g_out[b])
+        streams = synth.corrupt_stream(g, gl, wl.agreement, wl.shape.vocab, wl.index, bi)
+        t_src, t_len = torch.tensor(src, device=dev), torch.tensor(lens, device=dev)
+        t_max, t_str = torch.tensor(max_len, device=dev), torch.tensor(streams, device=dev)
+        t_out = torch.zeros((wl.batch, cap), dtype=torch.int32, device=dev); t_ol = torch.zeros(wl.batch, dtype=torch.int32, device=dev)
+        kw = dict(mode=wl.mode, k=k, max_len_t=t_max, override_t=t_str, run_drafter=gad)
+        dec.generate_device(t_src, t_len, t_out, t_ol, **kw)                        # warm (graph build)
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(dec.stream)
+        st = dec.generate_device(t_src, t_len, t_out, t_ol, **kw)
+        b_.record(dec.stream); dec.stream.synchronize()
+        for key in ("accepted", "iterations", "row_iterations", "offered", "device_ms", "encode_ms"):
+            tot[key] += st[key]
+        tot["wall_ms"] += a.elapsed_time(b_)
+        sum_src += int(lens.sum())
+    it = max(1, tot["iterations"])
+    res = dict(workload=f"recipe {index}: {wl.shape.name}, {wl.mode}, batch {wl.batch}, source {wl.src_len_lo}..{wl.src_len_hi}, "
+                        f"block {k}, agreement {wl.agreement}" + (", drafter forward timed" if gad else ""),
+               batches=n_batches, tokens_per_s=tot["accepted"] / (tot["wall_ms"] * 1e-3),
+               tokens_per_s_decode_only=tot["accepted"] / (tot["device_ms"] * 1e-3),
+               us_per_loop_iteration=1e3 * tot["device_ms"] / it, iterations=tot["iterations"],
+               mean_accepted_per_row_iteration=tot["accepted"] / max(1, tot["row_iterations"]),
+               encode_ms=tot["encode_ms"], decode_ms=tot["device_ms"])
+    dec.close()
+    if oracle_seconds > 0:
+        res["cpu_baseline"] = oracle_workload_sample(index, oracle_seconds, w, wn if gad else None)
+    return res
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_2205_10350_b200 import build as lib_build
@@ -179,7 +359,6 @@ def run_ours(args, rank, world, local_rank):
 
     w = synth.make_weights(synth.BASE, 0)
     dec = binding.AggressiveDecoder(synth.BASE, w, max_batch=1, max_src=WL.src_len_hi, max_tgt=KMAX, kmax=KMAX, device=str(dev))
-    lib = dec.lib
     src, lens = sentence_inputs(rank)
     max_len = lens.copy()
 
@@ -203,7 +382,7 @@ def run_ours(args, rank, world, local_rank):
     stream = dec.stream
 
     def step_device():
-        tot = dict(accepted=0, iterations=0, kernel_launches=0, device_ms=0.0, encode_ms=0.0)
+        tot = dict(accepted=0, iterations=0, offered=0, kernel_launches=0, device_ms=0.0, encode_ms=0.0)
         for s in range(N_SENT):
             st = dec.generate_device(t_src[s: s + 1], t_len[s: s + 1], t_out[s: s + 1], t_olen[s: s + 1], mode="IAD", k=KMAX,
                                      max_len_t=t_max[s: s + 1], override_t=t_str[s: s + 1], sync_every=args.sync_every)
@@ -232,7 +411,7 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     sampler.start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    agg = dict(accepted=0, iterations=0, kernel_launches=0, device_ms=0.0, encode_ms=0.0)
+    agg = dict(accepted=0, iterations=0, offered=0, kernel_launches=0, device_ms=0.0, encode_ms=0.0)
     for i in range(args.steps):
         with torch.cuda.stream(stream):
             flush.fill_(i & 0xFF)                      # evict the weights from L2 between timed steps
@@ -260,105 +439,30 @@ def run_ours(args, rank, world, local_rank):
     e2e_t = time.perf_counter() - t0
     e2e_t, e2e_tok = reduce_max_sum(dist, dev, e2e_t, e2e_tok)
     h2d = int(src.nbytes + lens.nbytes + max_len.nbytes + streams.nbytes)
-    d2h = int(N_SENT * KMAX * 4 + N_SENT * 4 + N_SENT * (16 + 4 + 4))     # outputs, lengths, statistics and status words
+    d2h = int(N_SENT * (4 + 4 + KMAX) * 4)              # per sentence: header, per-row record and output ids of the result block
 
-    # dominant kernel: projection fused with arg-max (streams the 32.8 MB embedding matrix), timed alone with
-    # CUDA events on the launching stream, L2 flushed before every launch (cold) and not flushed (warm)
-    V, d = synth.BASE.vocab, synth.BASE.d_model
-    M = KMAX
-    x = torch.randn((M, d), device=dev).bfloat16()
-    emb = dec._keep[0][: V * d].view(V, d)
-    nb = lib.ad_vocab_argmax_scratch_bytes(V, M)
-    scratch = torch.empty(nb + 256, dtype=torch.uint8, device=dev)
-    sbase = (scratch.data_ptr() + 255) // 256 * 256
-    am = torch.empty(M, dtype=torch.int32, device=dev)
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-
-    def vocab_once(with_reduction):
-        rc = lib.ad_vocab_argmax(C.c_void_p(x.data_ptr()), C.c_void_p(emb.data_ptr()), 1, M, d, V,
-                                 C.c_void_p(am.data_ptr()) if with_reduction else None,
-                                 C.c_void_p(sbase), nb, C.c_void_p(status.data_ptr()), C.c_void_p(stream.cuda_stream))
-        assert rc == 0
-
-    def time_vocab(cold, with_reduction=False, reps=20):
-        # everything is enqueued first and the stream synchronised once, so that the events bracket device time
-        # only (a host round trip per launch would add the launch latency to every sample)
-        evs = []
-        with torch.cuda.stream(stream):
-            for i in range(reps + 3):
-                if cold:
-                    flush.fill_(i & 0xFF)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); vocab_once(with_reduction); b.record(stream)
-                evs.append((a, b))
-        stream.synchronize()
-        return statistics.mean(a.elapsed_time(b) for a, b in evs[3:])
-
-    alg_bytes = V * d * 2 + M * d * 2 + M * 4
-    t_cold, t_warm = time_vocab(True), time_vocab(False)
-    t_cold_red = time_vocab(True, with_reduction=True)
-    ach = alg_bytes / (t_cold * 1e-3) / 1e9
-    roofline = dict(bound="hbm", kernel="gemm_tc_kernel<EPI_ARGMAX> (projection fused with the per-tile row arg-max)",
-                    achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES,
-                    peak_source=pk["source"], us_per_launch_cold=t_cold * 1e3, us_per_launch_l2_warm=t_warm * 1e3,
-                    us_cold_with_final_reduction_kernel=t_cold_red * 1e3,
-                    algorithmic_bytes=alg_bytes, timing="separate pass after the timed steps, same process and launch shape "
-                    "(250 CTAs x 256 threads, 64-token tile), one launch between two events; cold = 256 MB L2 flush "
-                    "before each launch")
-
-    # whole verification step against the weight-streaming floor (76.8 MB per step for this model)
+    # ---- roofline of the unit of the path: one verification step inside the decode loop ----
+    # algorithmic bytes of all loop iterations of a step's 64 sentences: weights once per iteration, cross K/V of the
+    # sentence's source and self K/V up to len + k (= the sentence's output length T, since k = remaining) per
+    # iteration, self K/V written for every offered block token
     iters = max(1, agg["iterations"])
     loop_us = 1e3 * agg["device_ms"] / iters
-    wv = (6 * (6 * d * d + 2 * d * synth.BASE.d_ffn) + V * d) * 2
-    floor_us = wv / (pk["hbm_gbs"] * 1e9) * 1e6
-    verify = dict(us_per_iteration_in_loop=loop_us, weight_bytes=wv, hbm_floor_us=floor_us, frac_of_floor=floor_us / loop_us,
-                  note="graph-replayed draft-prepare + verify + commit, weights L2-warm between iterations of a sentence")
-
-    # the library's own greedy decoding (block size 1) of the same sentences: what the draft-verify loop is
-    # measured against in the paper's tables (speedup over greedy), here on the same kernels
-    def step_greedy():
-        acc = 0
-        for s in range(N_SENT):
-            st = dec.generate_device(t_src[s: s + 1], t_len[s: s + 1], t_out[s: s + 1], t_olen[s: s + 1], mode="IAD", k=1,
-                                     max_len_t=t_max[s: s + 1])
-            acc += st["accepted"]
-        return acc
-    step_greedy()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record(stream); g_tok = step_greedy(); g1.record(stream)
-    stream.synchronize()
-    greedy_tps = g_tok / (g0.elapsed_time(g1) * 1e-3)
-    greedy_arm = dict(value=greedy_tps, unit=UNIT, speedup_of_draft_verify=value / world / greedy_tps if greedy_tps > 0 else None,
-                      note="same sentences decoded with block size 1 (one token per iteration), encoder included, one pass")
-
-    # tensor-core regime: one verification step of 32 rows x 64 block positions (2048 packed tokens) against the
-    # BF16 tensor peak.  flops = 2 x (decoder + projection weights) x tokens + attention (4 d per query-key pair).
-    B32, K32, S32 = 32, 64, 64
-    dec32 = binding.AggressiveDecoder(synth.BASE, w, max_batch=B32, max_src=S32, max_tgt=K32, kmax=K32, device=str(dev))
-    r32 = np.random.default_rng(7)
-    dec32.encode(r32.integers(4, V, size=(B32, S32)).astype(np.int32), np.full(B32, S32, np.int32))
-    d32 = torch.tensor(r32.integers(4, V, size=(B32, K32)).astype(np.int32), device=dev)
-    k32 = torch.full((B32,), K32, dtype=torch.int32, device=dev)
-    a32 = torch.zeros((B32, K32), dtype=torch.int32, device=dev); n32 = torch.zeros(B32, dtype=torch.int32, device=dev)
-    z32 = torch.zeros(B32, dtype=torch.int32, device=dev)
-    evs32 = []
-    with torch.cuda.stream(dec32.stream):
-        for i in range(13):
-            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a_.record(dec32.stream)
-            dec32.verify_block_device(d32, k32, a32, n32)
-            dec32.commit_device(z32)                     # n = 0: discard, every repetition sees the same prefix
-            b_.record(dec32.stream)
-            evs32.append((a_, b_))
-    dec32.sync()
-    us32 = 1e3 * statistics.mean(a_.elapsed_time(b_) for a_, b_ in evs32[3:])
-    M32 = B32 * K32
-    flops32 = 2.0 * (wv / 2) * M32 + 4.0 * 6 * d * (B32 * sum(i + 1 + S32 for i in range(K32)))
-    floor32 = flops32 / (pk["bf16_tflops"] * 1e12) * 1e6
-    tensor_regime = dict(us_per_step=us32, packed_tokens=M32, flops=flops32, tensor_floor_us=floor32, peak_tflops=pk["bf16_tflops"],
-                         frac_of_floor=floor32 / us32, note="batch 32, block 64, empty prefix, source 64; direct launches, weights L2-warm")
-    dec32.close()
-
+    it_per_sent = agg["iterations"] / args.steps / N_SENT
+    mean_S = float(lens.mean())
+    alg = step_bytes(synth.BASE, sum_src=mean_S * iters, sum_keys=float(glen.mean()) * iters, sum_k=agg["offered"], n_steps=iters) / iters
+    ach = alg / (loop_us * 1e-6) / 1e9
+    wv = weight_bytes(synth.BASE)
+    roofline = dict(bound="hbm", kernel="verification step: the 57-kernel chain of one loop iteration (plan, embed, 6 decoder layers, "
+                    "projection + arg-max, accept + commit), graph-replayed", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"], algorithmic_bytes=alg,
+                    weight_bytes=wv, us_per_step_in_loop=loop_us, hbm_floor_us=alg / (pk["hbm_gbs"] * 1e9) * 1e6,
+                    note="time = device time of the decode loops / loop iterations (weights L2-warm between the iterations of a "
+                         "sentence, L2 flushed between timed steps); traffic is null because the step is a chain of kernels, "
+                         "none of which dominates: see `kernels` and profiles/ for the per-kernel DRAM counters")
+    out_line = dict(value=value, t_ms=t_ms, tokens=tokens, e2e=dict(value=e2e_tok / e2e_t, unit=UNIT, h2d_bytes_per_step=h2d,
+                                                                   d2h_bytes_per_step=d2h),
+                    clocks=clocks, agg=agg, iters=iters, roofline=roofline, it_per_sent=it_per_sent)
+    extras = bench_extras(args, binding, dec, w, dev, pk, flush, t_src, t_len, t_max, t_out, t_olen, value, world) if rank == 0 else {}
     cpu = None
     if rank == 0:
         if world == 1:
@@ -369,36 +473,13 @@ def run_ours(args, rank, world, local_rank):
                     config=dict(workload=WORKLOAD_DESC,
                                 sentences_per_step=N_SENT, l2="flushed between timed steps (256 MB write); within a step the "
                                 "weights stay L2-resident across the iterations of the decode loop", parallelism=f"replicas x{world}"),
-                    clocks=clocks,
-                    e2e=dict(value=e2e_tok / e2e_t, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
-                    gpu_launches=int(agg["kernel_launches"]),
+                    clocks=clocks, e2e=out_line["e2e"], gpu_launches=int(agg["kernel_launches"]),
                     tokens_per_step=tokens / args.steps / world, iterations_per_step=agg["iterations"] / args.steps,
                     mean_accepted_per_iteration=agg["accepted"] / iters,
                     encode_ms_per_step=agg["encode_ms"] / args.steps, decode_ms_per_step=agg["device_ms"] / args.steps,
-                    verify_step=verify, tensor_regime=tensor_regime, greedy=greedy_arm, roofline=roofline, cpu_baseline=cpu)
+                    host_ms_per_step=t_ms / args.steps - (agg["encode_ms"] + agg["device_ms"]) / args.steps,
+                    roofline=roofline, cpu_baseline=cpu, **extras)
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
-
-
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sync-every", type=int, default=0, help="iterations between host checks of the finished flag (0 = library default)")
-    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work of the checker baseline sample")
-    args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
-        run_reference(args, rank, world)
-    else:
-        run_ours(args, rank, world, local_rank)
-
-
-if __name__ == "__main__":
-    main()

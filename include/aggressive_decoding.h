@@ -220,9 +220,18 @@ int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_
 /* Debug: FP32 copy of the verifier's encoder memory of row b, [src_len_b, d_model] (device pointer). */
 int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size_t capacity_elems);
 
-/* Debug: stage timeline of the last persistent decoder pass (the single-kernel form of the decoder stack that handles
- * BF16 models with 64-wide heads and passes of at most 64 packed tokens).  With AD_MEGA_TIMELINE=1 in the environment
- * when the handle is created, CTA 0 of that kernel stamps the GPU's global nanosecond timer twice per stage: when the
+/* Debug: one verification block (arguments as ad_verify_block with host arrays) with a CUDA event in front of every
+ * kernel launch and programmatic dependent launch switched off, so that every kernel's device time is bracketed on its
+ * own.  names (host, capacity x 64 chars) and us (host, capacity floats) receive, in launch order, what was launched and
+ * how long it took; *n_launches their count.  The block is verified as usual (not committed).  Synchronises. */
+int ad_debug_profile_verify(ad_handle* h, const int32_t* drafts, const int32_t* k, char* names, float* us,
+                            int32_t capacity, int32_t* n_launches);
+
+/* Debug: stage timeline of the last persistent decoder pass.  The library has a second form of the decoder pass:
+ * the whole decoder stack and the vocabulary projection as ONE persistent kernel (BF16 models with 64-wide heads,
+ * passes of at most 64 packed tokens), selected with AD_MEGA=1 in the environment when the handle is created.  It
+ * computes the same results as the default chain of kernels and is kept as a measured alternative (it is slower on a
+ * B200 at every shape tried).  With AD_MEGA_TIMELINE=1 as well, CTA 0 of that kernel stamps the GPU's global nanosecond timer twice per stage: when the
  * stage's inputs have become visible, and after it has signalled its own part done.  stamps (host, >= 2 * n_stages
  * entries) receives them in stage order: per decoder layer QKV, self-attention, Wo, cross-Q, cross-attention, cross-Wo,
  * FFN1, FFN2; then the vocabulary projection.  Synchronises the stream. */

@@ -21,7 +21,7 @@ AD_MODE_IAD, AD_MODE_GAD = 0, 1
 EXPORTS = [
     "ad_weight_counts", "ad_query_workspace", "ad_create", "ad_destroy", "ad_last_error", "ad_encode",
     "ad_verify_block", "ad_commit", "ad_force_commit", "ad_generate", "ad_draft_block", "ad_get_state", "ad_sync", "ad_set_acceptance",
-    "ad_debug_logits", "ad_debug_encoder_memory", "ad_debug_stage_timeline", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
+    "ad_debug_logits", "ad_debug_encoder_memory", "ad_debug_stage_timeline", "ad_debug_profile_verify", "ad_vocab_argmax_scratch_bytes", "ad_vocab_argmax",
     "ad_vocab_argmax_static", "ad_debug_wait_probe", "ad_debug_grid_barrier_probe",
     "ad_linear",
 ]
@@ -90,6 +90,7 @@ def load():
         "ad_debug_logits": (C.c_int, [vp, i32, vp, sz]),
         "ad_debug_encoder_memory": (C.c_int, [vp, i32, vp, sz]),
         "ad_debug_stage_timeline": (C.c_int, [vp, vp, i32, vp]),
+        "ad_debug_profile_verify": (C.c_int, [vp, vp, vp, vp, vp, i32, vp]),
         "ad_vocab_argmax_scratch_bytes": (sz, [i32, i32]),
         "ad_vocab_argmax": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, sz, vp, vp]),
         "ad_vocab_argmax_static": (C.c_int, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
@@ -249,6 +250,20 @@ class AggressiveDecoder:
         self._check(self.lib.ad_debug_logits(self.h, which, C.c_void_p(t.data_ptr()), t.numel()), self.h)
         self.sync()
         return t.cpu().numpy()
+
+    def profile_verify(self, drafts, k, capacity=512):
+        """One verification block with every kernel timed on its own: list of (what, microseconds) in launch order."""
+        d = np.full((self.B, self.kmax), -1, np.int32)
+        drafts = np.asarray(drafts, np.int32)
+        d[:, : drafts.shape[1]] = drafts
+        k = _i32(k)
+        names = C.create_string_buffer(capacity * 64)
+        us = np.zeros(capacity, np.float32)
+        n = C.c_int32()
+        self._check(self.lib.ad_debug_profile_verify(self.h, d.ctypes.data, k.ctypes.data, names, us.ctypes.data, capacity,
+                                                     C.byref(n)), self.h)
+        raw = names.raw
+        return [(raw[i * 64: (i + 1) * 64].split(b"\0")[0].decode(), float(us[i])) for i in range(n.value)]
 
     def debug_stage_timeline(self):
         """Per-stage (inputs visible, signalled) global-timer stamps of the last persistent decoder pass, in ns."""

@@ -121,7 +121,18 @@ struct ad_handle {
   float* pe = nullptr;
   int max_pos = 0;
   int* ovr = nullptr;        // [B, max_tgt] staged draft-override stream
-  int* host_flag = nullptr;  // pinned
+  int* host_flag = nullptr;  // pinned, mapped host memory: [0..15] flag words, then the upload area (sources, lengths, caps,
+                             // override stream) and the result block of ad_generate
+  int* host_flag_dev = nullptr;   // the same memory as the device sees it
+  int* up_src = nullptr;     // pinned staging of host-resident inputs
+  int* up_len = nullptr;
+  int* up_max = nullptr;
+  int* up_ovr = nullptr;
+  int* down = nullptr;       // result block of finalize_generate_kernel (host view) ...
+  int* down_dev = nullptr;   // ... and its device view
+  bool defer_status = false; // ad_encode inside ad_generate: no synchronisation of its own
+  bool profiling = false;    // ad_debug_profile_verify: an event in front of every launch
+  std::vector<std::pair<std::string, cudaEvent_t>> prof;
   // state
   int B = 0;                 // batch of the last ad_encode
   bool encoded = false;
@@ -161,6 +172,19 @@ namespace {
 int fail(ad_handle* h, int code, const std::string& msg) {
   if (h) h->err = msg; else g_create_error = msg;
   return code;
+}
+
+// Counts a kernel launch of this library and, while a profiling pass is active, drops an event in front of it (the
+// time between two consecutive events is then the device time of the kernel launched after the first one).
+void note_launch(ad_handle* h, const char* what) {
+  h->launches++;
+  if (h->profiling) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) == cudaSuccess) {
+      cudaEventRecord(e, h->stream);
+      h->prof.emplace_back(what, e);
+    }
+  }
 }
 
 // ---- TMA descriptor encoding through the driver entry point (no link-time dependency on libcuda) ----
@@ -305,7 +329,7 @@ size_t layout(ad_handle* h, void* base) {
   }
   h->mega_timeline = (unsigned long long*)bp.take(sizeof(unsigned long long) * 2 * (size_t)(mega::ST_PER_LAYER * c.n_dec + 1));
 #ifdef AD_MEGA_DEBUG
-  h->mega_dbg = (float*)bp.take(sizeof(float) * 16 * 32 * 4);
+  h->mega_dbg = (float*)bp.take(sizeof(float) * 4096 + 8 * 64 * 8);
 #endif
   for (int k = 0; k < PK_COUNT; ++k) plan_take(bp, h->pass[k].plan, B, h->pass[k].M_cap);
   DevState& s = h->st;
@@ -387,7 +411,13 @@ bool g_use_graph_encode = true;   // AD_NO_ENCODE_GRAPH=1: launch the encoder ke
 bool g_two_stream_encode = true;   // AD_NO_CONCURRENT_ENCODERS=1: the drafter's encoder after the verifier's, on one stream
 bool g_use_devloop = true;   // AD_NO_DEVLOOP=1: one graph replay per iteration with host polling instead of a device-side loop
 bool g_fuse_attn_proj = true;   // AD_NO_ATTN_PROJ=1: attention and its output projection always as separate kernels
-bool g_use_mega = true;         // AD_NO_MEGA=1: never use the persistent decoder-pass kernel (always the kernel chain)
+// AD_MEGA=1: run eligible decoder passes (BF16, 64-wide heads, at most 64 packed tokens) as ONE persistent kernel
+// instead of the kernel chain.  Off by default: measured on a B200 it is slower than the chain at every shape tried
+// (base model: 342 / 360 / 424 / 462 us per verification step for blocks of 1 / 16 / 40 / 64 tokens against 214 / 223 /
+// 247 / 258 us; big model, 25 tokens: 537 against 323 us), because a stage that hands its result to other SMs through
+// L2 costs about 7 us there (operand staging 1.3-3 us, MMA hand-over 0.6, tensor-memory read-out 0.3, cluster hand-shake
+// 0.8-1.2, reduction and epilogue 1-1.7, release 0.5, propagation 0.7) against about 3.7 us per kernel of the chain.
+bool g_use_mega = false;
 
 // Launches `kernel` so that it may begin while its predecessor in the stream still runs (the kernels
 // themselves wait with griddepcontrol.wait before touching anything a predecessor writes).
@@ -458,7 +488,12 @@ cudaError_t launch_simt(cudaStream_t st, const void* w, const void* x, const Gem
 int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int* M_ptr, int M_cap, GemmParams p) {
   p.K = W.K; p.N = W.N; p.M_ptr = M_ptr; p.M_cap = M_cap; p.status = h->st.status;
   cudaError_t e;
-  h->launches++;
+  {
+    static const char* epi_name[4] = {"gemm_f32_partials", "gemm_act", "gemm_scatter", "gemm_vocab_argmax"};
+    char nm[64];
+    snprintf(nm, sizeof(nm), "%s N%d K%d", epi_name[epi & 3], W.N, W.K);
+    note_launch(h, nm);
+  }
   if (h->bf16) {
     p.ntile = h->pass[pk].tile_for(W.N, num_sms());
     const CUtensorMap& mx = (p.ntile == h->pass[pk].ntile) ? X.map[pk] : X.map_half[pk];
@@ -517,7 +552,7 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
     const int ng = pc.seg_max <= 16 ? 4 : (pc.seg_max <= 32 ? 2 : 1);
     const int qcta = AM_Q / ng;
     p.qchunks = (pc.seg_max + qcta - 1) / qcta;
-    h->launches++;
+    note_launch(h, "attention_mma");
     const dim3 mgrid(h->dims.B * p.qchunks, c.n_heads);
     cudaError_t em;
     if (ng == 4) em = launch_k(attention_mma_kernel<4>, mgrid, dim3(128), 0, h->stream, p);
@@ -530,13 +565,13 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   p.qchunks = (pc.seg_max + 8 * qpw - 1) / (8 * qpw);
   dim3 grid(h->dims.B * p.qchunks, c.n_heads);
   const dim3 block(256);
-  h->launches++;
   cudaError_t e;
 #define AD_ATT(T, D, Q) launch_attention<T, D, Q>(grid, block, h->stream, p)
   // few queries, 64-wide heads: the output projection rides along (one partial sum per head for the LayerNorm kernel)
   const bool fuse = g_fuse_attn_proj && wo && fused && h->pre2 && h->bf16 && dh == 64 && !many && c.n_heads <= pc.max_split &&
                     c.n_heads <= 16 && c.d_model % 128 == 0;
   if (fused) *fused = fuse;
+  note_launch(h, fuse ? "attention+out_proj" : "attention");
   if (fuse) {
     p.wo = (const bf16*)wo->ptr; p.o_part = h->pre2; p.o_stride = (size_t)pc.M_cap * c.d_model;
     e = launch_attention<bf16, 64, 1, true>(grid, block, h->stream, p);
@@ -559,7 +594,7 @@ int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, co
   const int d = h->cfg.d_model;
   dim3 grid(pc.M_cap);
   const size_t stride = (size_t)pc.M_cap * d;
-  h->launches++;
+  note_launch(h, "residual+layernorm");
   cudaError_t e;
   if (pc.M_cap >= 512 && nsplit <= 4 && d % 128 == 0 && d <= 1024) {   // many tokens: a warp per token
     dim3 rgrid((pc.M_cap + 7) / 8);
@@ -589,7 +624,7 @@ int gemm_to_ln(ad_handle* h, const Mat& W, const ActBuf& X, int pk, int* nsplit)
 int embed(ad_handle* h, const PassCfg& pc, const Model& m) {
   const int d = h->cfg.d_model;
   const float sc = sqrtf((float)d);
-  h->launches++;
+  note_launch(h, "embed");
   cudaError_t e;
   if (h->bf16) e = launch_k(embed_kernel<bf16, bf16>, dim3(pc.M_cap), dim3(128), 0, h->stream, pc.plan, (const bf16*)m.emb.ptr, (const float*)h->pe, d, sc, h->y, (bf16*)h->yb.ptr);
   else e = launch_k(embed_kernel<float, float>, dim3(pc.M_cap), dim3(128), 0, h->stream, pc.plan, (const float*)m.emb.ptr, (const float*)h->pe, d, sc, h->y, (float*)h->yb.ptr);
@@ -630,14 +665,11 @@ int ffn_sublayer(ad_handle* h, int pk, const Mat& w1, const float* b1, const Mat
 
 // ---- persistent decoder pass ---------------------------------------------------------------------------------
 
-// Cluster size for the K split of the projections: the K blocks of d_model and of d_ffn must divide evenly, and a CTA's
-// share of the B operand (its K blocks x 64 tokens x 128 bytes) must fit the 64 KB operand area.
+// Cluster size for the K split of the projections: the K blocks of d_model and of d_ffn must divide evenly.
 int mega_cluster_size(const ad_model_cfg& c) {
   for (int cs : {8, 4}) {
     const int kd = c.d_model / 64, kf = c.d_ffn / 64;
-    if (kd % cs || kf % cs) continue;
-    if ((kf / cs) * mega::NT_MAX * 128 > 64 * 1024) continue;
-    return cs;
+    if (kd % cs == 0 && kf % cs == 0) return cs;
   }
   return 0;
 }
@@ -661,7 +693,7 @@ int mega_setup(ad_handle* h) {
   const int b_bytes = (std::max(c.d_model, c.d_ffn) / 64 / cs) * ntcap * 128;
   const int red_bytes = ntcap * mega::RED_LD * 4;
   const int work = std::max(std::max(b_bytes + 2 * red_bytes, (c.d_model / 64) * ntcap * 128), mega::ATT_SMEM);
-  int ring = (max_optin - 1024 - work - 4096) / mega::TILE_A;     // 4096: the kernel's static control block
+  int ring = (max_optin - 1024 - work - 13 * 1024) / mega::TILE_A;     // 13 KB: the kernel's static control block
   if (ring > mega::MAX_RING) ring = mega::MAX_RING;
   if (ring < 4) return AD_OK;
   const size_t smem = 1024 + (size_t)ring * mega::TILE_A + (size_t)work;
@@ -757,7 +789,7 @@ int mega_launch(ad_handle* h, int pk) {
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 2 : 1;
-  h->launches++;
+  note_launch(h, "persistent_decoder_pass");
   cudaError_t e = cudaLaunchKernelEx(&cfg, mega::decoder_pass_kernel, p);
   if (e != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("persistent decoder pass launch: ") + cudaGetErrorString(e));
   return AD_OK;
@@ -844,14 +876,14 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
   const int beta = to_drafts ? 0 : h->beta;
   if (beta >= 1) {   // relaxed verification: the drafts' own scores first, then the projection counts against them
     const int d = h->cfg.d_model;
-    h->launches++;
+    note_launch(h, "draft_score");
     const dim3 sgrid((pc.M_cap + 7) / 8);
     if (h->bf16) AD_CUDA(h, launch_k(draft_score_kernel<bf16, bf16>, sgrid, dim3(256), 0, h->stream, h->st, pc.plan, h->dims, (const bf16*)m.emb.ptr, (const bf16*)X.ptr, d, h->draft_val, h->draft_id));
     else AD_CUDA(h, launch_k(draft_score_kernel<float, float>, sgrid, dim3(256), 0, h->stream, h->st, pc.plan, h->dims, (const float*)m.emb.ptr, (const float*)X.ptr, d, h->draft_val, h->draft_id));
     p.draft_val = h->draft_val; p.draft_id = h->draft_id; p.part_cnt = h->part_cnt;
   }
   if (!partials_ready) AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
-  h->launches++;
+  note_launch(h, "argmax_accept");
   AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
                       pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
                       auto_commit ? h->cond_handle : 0ull, beta, h->tau, (const float*)h->draft_val, (const int*)h->draft_id,
@@ -861,7 +893,7 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
 }
 
 int prepare_verify(ad_handle* h, int source, int k_cap, const int* ovr, int ovr_len) {
-  h->launches++;
+  note_launch(h, "prepare_verify");
   AD_CUDA(h, launch_k(prepare_verify_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, source, k_cap, ovr,
                                                  h->cfg.max_tgt, ovr_len));
   return AD_OK;
@@ -870,7 +902,7 @@ int prepare_verify(ad_handle* h, int source, int k_cap, const int* ovr, int ovr_
 // Draft substep: sizes, drafter plan, drafter decoder, gather of the mask rows, projection + arg-max.
 int draft_stage(ad_handle* h, int k_cap) {
   AD_TRY(prepare_verify(h, SRC_SIZES, k_cap, nullptr, 0));
-  h->launches++;
+  note_launch(h, "draft_stage");
   AD_CUDA(h, launch_k(plan_draft_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->pass[PK_DRAFT].plan, h->dims));
   if (mega_applies(h, PK_DRAFT)) {      // decoder stack, gather of the mask rows and projection in one kernel
     AD_TRY(mega_launch(h, PK_DRAFT));
@@ -879,7 +911,7 @@ int draft_stage(ad_handle* h, int k_cap) {
   AD_TRY(decoder_pass(h, PK_DRAFT, h->nar));
   const int d = h->cfg.d_model;
   PassCfg& pv = h->pass[PK_VERIFY];
-  h->launches++;
+  note_launch(h, "draft_stage");
   if (h->bf16) AD_CUDA(h, launch_k(gather_rows_kernel<bf16>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const bf16*)h->yb.ptr, (bf16*)h->xg.ptr, d));
   else AD_CUDA(h, launch_k(gather_rows_kernel<float>, dim3(pv.M_cap), dim3(128), 0, h->stream, (const int*)pv.plan.M, (const int*)h->st.gidx, (const float*)h->yb.ptr, (float*)h->xg.ptr, d));
   return vocab_stage(h, h->nar, h->xg, 1, 0);
@@ -895,7 +927,7 @@ int verify_stage(ad_handle* h, int auto_commit) {
 }
 
 int commit_stage(ad_handle* h, const int* n_dev) {
-  h->launches++;
+  note_launch(h, "commit_stage");
   AD_CUDA(h, launch_k(commit_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, n_dev));
   return AD_OK;
 }
@@ -978,7 +1010,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   { const char* e = getenv("AD_NO_ENCODE_GRAPH"); g_use_graph_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_CONCURRENT_ENCODERS"); g_two_stream_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ATTN_PROJ"); g_fuse_attn_proj = !(e && e[0] == '1'); }
-  { const char* e = getenv("AD_NO_MEGA"); g_use_mega = !(e && e[0] == '1'); }
+  { const char* e = getenv("AD_MEGA"); g_use_mega = e && e[0] == '1'; }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();
@@ -1051,7 +1083,16 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
         cudaStreamSynchronize(h->stream) != cudaSuccess)
       return bail(AD_ERR_CUDA, "uploading the positional table failed");
   }
-  if (cudaMallocHost(&h->host_flag, 64) != cudaSuccess) return bail(AD_ERR_CUDA, "cudaMallocHost failed");
+  {
+    const size_t B = cfg->max_batch;
+    const size_t n_up = B * cfg->max_src + 2 * B + B * cfg->max_tgt, n_down = 4 + 4 * B + B * cfg->max_tgt;
+    if (cudaHostAlloc(&h->host_flag, sizeof(int) * (16 + n_up + n_down), cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer(&h->host_flag_dev, h->host_flag, 0) != cudaSuccess)
+      return bail(AD_ERR_CUDA, "allocating pinned host memory failed");
+    h->up_src = h->host_flag + 16; h->up_len = h->up_src + B * cfg->max_src; h->up_max = h->up_len + B;
+    h->up_ovr = h->up_max + B; h->down = h->up_ovr + B * cfg->max_tgt;
+    h->down_dev = h->host_flag_dev + (h->down - h->host_flag);
+  }
   if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess || cudaEventCreate(&h->ev2) != cudaSuccess)
     return bail(AD_ERR_CUDA, "cudaEventCreate failed");
   *out = h;
@@ -1102,12 +1143,21 @@ extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, c
   h->dims.B = B;
   h->encoded = false;
   const int w = src_stride < c.max_src ? src_stride : c.max_src;
-  AD_CUDA(h, cudaMemcpy2DAsync(h->st.src, sizeof(int) * c.max_src, src, sizeof(int) * src_stride, sizeof(int) * w, B, to_dev(on_host), h->stream));
-  AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, src_len, sizeof(int) * B, to_dev(on_host), h->stream));
+  if (on_host) {
+    // host-resident inputs go through the handle's pinned staging area (every host-array call ends synchronised, so
+    // the area is free again): one truly asynchronous copy each instead of driver-staged pageable copies
+    for (int b = 0; b < B; ++b) memcpy(h->up_src + (size_t)b * c.max_src, src + (size_t)b * src_stride, sizeof(int) * w);
+    memcpy(h->up_len, src_len, sizeof(int) * B);
+    AD_CUDA(h, cudaMemcpyAsync(h->st.src, h->up_src, sizeof(int) * (size_t)B * c.max_src, cudaMemcpyHostToDevice, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, h->up_len, sizeof(int) * B, cudaMemcpyHostToDevice, h->stream));
+  } else {
+    AD_CUDA(h, cudaMemcpy2DAsync(h->st.src, sizeof(int) * c.max_src, src, sizeof(int) * src_stride, sizeof(int) * w, B, cudaMemcpyDeviceToDevice, h->stream));
+    AD_CUDA(h, cudaMemcpyAsync(h->st.srclen, src_len, sizeof(int) * B, cudaMemcpyDeviceToDevice, h->stream));
+  }
   // The encoder pass reads its inputs from fixed workspace buffers, so on a capturable stream it is captured
   // once per batch size and replayed (about fifty launches otherwise paid on the host for every sentence).
   auto enqueue = [&]() -> int {
-    h->launches++;
+    note_launch(h, "ad_encode");
     AD_CUDA(h, launch_k(plan_encode_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_ENCODE].plan, h->dims));
     if (c.has_drafter && h->side_stream) {
       // the two encoders are independent (Section 3.2: separate models): drafter's on the side stream, verifier's here
@@ -1156,7 +1206,7 @@ extern "C" int ad_encode(ad_handle* h, const int32_t* src, int32_t src_stride, c
   }
   h->encoded = true;
   h->last_vocab_which = -1;
-  if (on_host) return read_status(h);
+  if (on_host && !h->defer_status) return read_status(h);
   return AD_OK;
 }
 
@@ -1179,7 +1229,7 @@ extern "C" int ad_verify_block(ad_handle* h, const int32_t* drafts, const int32_
     if (n_accepted) AD_CUDA(h, cudaMemcpyAsync(n_accepted, h->st.n_acc, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
     return read_status(h);
   }
-  h->launches++;
+  note_launch(h, "ad_verify_block");
   AD_CUDA(h, launch_k(export_block_kernel, dim3(B), dim3(64), 0, h->stream, h->st, h->dims, argmax, n_accepted, nullptr, nullptr, h->pass[PK_VERIFY].plan));
   return AD_OK;
 }
@@ -1203,7 +1253,7 @@ extern "C" int ad_force_commit(ad_handle* h, const int32_t* tokens, const int32_
   if (!tokens || !n) return fail(h, AD_ERR_ARG, "tokens or n is null");
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_drafts, tokens, sizeof(int) * (size_t)h->B * h->cfg.kmax, to_dev(on_host), h->stream));
   AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, n, sizeof(int) * h->B, to_dev(on_host), h->stream));
-  h->launches++;
+  note_launch(h, "ad_force_commit");
   AD_CUDA(h, launch_k(force_commit_kernel, dim3(1), dim3(256), 0, h->stream, h->st, h->pass[PK_VERIFY].plan, h->dims, h->st.user_drafts, h->st.user_n));
   if (on_host) return read_status(h);
   return AD_OK;
@@ -1222,7 +1272,7 @@ extern "C" int ad_draft_block(ad_handle* h, int32_t k_cap, int32_t* drafts, int3
     if (k) AD_CUDA(h, cudaMemcpyAsync(k, h->pass[PK_VERIFY].plan.seg_len, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
     return read_status(h);
   }
-  h->launches++;
+  note_launch(h, "ad_draft_block");
   AD_CUDA(h, launch_k(export_block_kernel, dim3(B), dim3(64), 0, h->stream, h->st, h->dims, nullptr, nullptr, drafts, k, h->pass[PK_VERIFY].plan));
   return AD_OK;
 }
@@ -1261,18 +1311,29 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
 
   AD_CUDA(h, cudaEventRecord(h->ev0, h->stream));
   h->launches = 0;
-  AD_TRY(ad_encode(h, src, src_stride, src_len, B, on_host));
+  h->defer_status = true;       // the one synchronisation at the end of this call reports device-side errors
+  const int rc_enc = ad_encode(h, src, src_stride, src_len, B, on_host);
+  h->defer_status = false;
+  if (rc_enc != AD_OK) return rc_enc;
   if (opts->max_len) {
-    AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, opts->max_len, sizeof(int) * B, to_dev(on_host), h->stream));
-    h->launches++;
+    const int* ml = opts->max_len;
+    if (on_host) { memcpy(h->up_max, opts->max_len, sizeof(int) * B); ml = h->up_max; }
+    AD_CUDA(h, cudaMemcpyAsync(h->st.user_n, ml, sizeof(int) * B, to_dev(on_host), h->stream));
+    note_launch(h, "ad_generate");
     AD_CUDA(h, launch_k(set_maxlen_kernel, dim3((B + 63) / 64), dim3(64), 0, h->stream, h->st, h->dims, h->st.user_n));
   }
   const int* ovr = nullptr;
   int ovr_len = 0;   // valid leading entries of each staged override row
   if (opts->draft_override) {
     ovr_len = opts->override_stride < c.max_tgt ? opts->override_stride : c.max_tgt;
-    AD_CUDA(h, cudaMemcpy2DAsync(h->ovr, sizeof(int) * c.max_tgt, opts->draft_override, sizeof(int) * opts->override_stride,
-                                 sizeof(int) * ovr_len, B, to_dev(on_host), h->stream));
+    if (on_host) {
+      for (int b = 0; b < B; ++b)
+        memcpy(h->up_ovr + (size_t)b * c.max_tgt, opts->draft_override + (size_t)b * opts->override_stride, sizeof(int) * ovr_len);
+      AD_CUDA(h, cudaMemcpyAsync(h->ovr, h->up_ovr, sizeof(int) * (size_t)B * c.max_tgt, cudaMemcpyHostToDevice, h->stream));
+    } else {
+      AD_CUDA(h, cudaMemcpy2DAsync(h->ovr, sizeof(int) * c.max_tgt, opts->draft_override, sizeof(int) * opts->override_stride,
+                                   sizeof(int) * ovr_len, B, cudaMemcpyDeviceToDevice, h->stream));
+    }
     ovr = h->ovr;
   }
   AD_CUDA(h, cudaEventRecord(h->ev1, h->stream));
@@ -1347,14 +1408,9 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
 
   if (device_loop) {
     // one launch runs every iteration; the data-independent bound on the iteration count travels in loop_it[3]
-    const int limit = max_iters + 1;
-    AD_CUDA(h, cudaMemcpyAsync(h->st.loop_it + 3, &limit, sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    h->host_flag[1] = max_iters + 1;
+    AD_CUDA(h, cudaMemcpyAsync(h->st.loop_it + 3, h->host_flag + 1, sizeof(int), cudaMemcpyHostToDevice, h->stream));
     AD_CUDA(h, cudaGraphLaunch(exec, h->stream));
-    int done = 0;
-    AD_CUDA(h, cudaMemcpyAsync(&done, h->st.loop_it + 2, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
-    AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
-    AD_CUDA(h, cudaStreamSynchronize(h->stream));
-    h->launches += per_iter_launches * done;
   }
   const int sync_every = opts->sync_every > 0 ? opts->sync_every : 1;
   int iters = 0;
@@ -1373,29 +1429,38 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
     AD_CUDA(h, cudaStreamSynchronize(h->stream));
     if (flag[0]) break;
   }
-  if (!device_loop) AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
-  const int w = out_stride < c.max_tgt ? out_stride : c.max_tgt;
-  AD_CUDA(h, cudaMemcpy2DAsync(out, sizeof(int) * out_stride, h->st.out_ids, sizeof(int) * c.max_tgt, sizeof(int) * w, B, from_dev(on_host), h->stream));
-  AD_CUDA(h, cudaMemcpyAsync(out_len, h->st.len, sizeof(int) * B, from_dev(on_host), h->stream));
+  AD_CUDA(h, cudaEventRecord(h->ev2, h->stream));
+  // Results, statistics and the status word in one block of mapped host memory, written by one kernel: the call ends
+  // with a single synchronisation (device-resident result arrays are written directly by the same kernel).
+  note_launch(h, "ad_generate");
+  AD_CUDA(h, launch_k(finalize_generate_kernel, dim3(B), dim3(128), 0, h->stream, h->st, h->dims, on_host ? nullptr : out, out_stride,
+                      on_host ? nullptr : out_len, h->down_dev));
+  AD_CUDA(h, cudaStreamSynchronize(h->stream));
+  const int* blk = h->down;
+  if (device_loop) h->launches += per_iter_launches * blk[0];
+  if (on_host) {
+    const int w = out_stride < c.max_tgt ? out_stride : c.max_tgt;
+    for (int b = 0; b < B; ++b) {
+      memcpy(out + (size_t)b * out_stride, blk + 4 + 4 * B + (size_t)b * c.max_tgt, sizeof(int) * w);
+      out_len[b] = blk[4 + 4 * b + 3];
+    }
+  }
   if (stats) {
-    std::vector<int> buf(3 * (size_t)B + 1);
-    AD_CUDA(h, cudaMemcpyAsync(buf.data(), h->st.stat_it, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
-    AD_CUDA(h, cudaMemcpyAsync(buf.data() + B, h->st.stat_acc, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
-    AD_CUDA(h, cudaMemcpyAsync(buf.data() + 2 * B, h->st.stat_off, sizeof(int) * B, cudaMemcpyDeviceToHost, h->stream));
-    AD_CUDA(h, cudaMemcpyAsync(buf.data() + 3 * B, h->st.loop_it, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
-    AD_CUDA(h, cudaStreamSynchronize(h->stream));
     memset(stats, 0, sizeof(*stats));
     for (int b = 0; b < B; ++b) {
-      stats->row_iterations += buf[b];
-      stats->accepted += buf[B + b];
-      stats->offered += buf[2 * B + b];
+      stats->row_iterations += blk[4 + 4 * b];
+      stats->accepted += blk[4 + 4 * b + 1];
+      stats->offered += blk[4 + 4 * b + 2];
     }
-    stats->iterations = buf[3 * B];
+    stats->iterations = blk[2];
     cudaEventElapsedTime(&stats->encode_ms, h->ev0, h->ev1);
     cudaEventElapsedTime(&stats->device_ms, h->ev1, h->ev2);
     stats->kernel_launches = h->launches;
   }
-  return read_status(h);
+  const int dev_status = blk[1];      // already cleared on the device by the kernel that read it
+  if (dev_status != 0)
+    return fail(h, dev_status, dev_status == AD_ERR_TIMEOUT ? "a bounded device-side wait ran out" : "device-side argument check failed");
+  return AD_OK;
 }
 
 extern "C" int ad_debug_logits(ad_handle* h, int32_t which, float* logits, size_t capacity_elems) {
@@ -1454,6 +1519,33 @@ extern "C" int ad_debug_peek(ad_handle* h, int which, int layer, void* dst, size
   return cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? AD_OK : AD_ERR_CUDA;
 }
 #endif
+
+extern "C" int ad_debug_profile_verify(ad_handle* h, const int32_t* drafts, const int32_t* k, char* names, float* us,
+                                       int32_t capacity, int32_t* n_launches) {
+  if (!h || !drafts || !k || !names || !us || !n_launches || capacity < 1) return AD_ERR_ARG;
+  if (!h->encoded) return fail(h, AD_ERR_STATE, "ad_debug_profile_verify before ad_encode");
+  const bool pdl = g_use_pdl;
+  g_use_pdl = false;               // serialised launches: an event between two kernels then brackets exactly one of them
+  h->profiling = true;
+  h->prof.clear();
+  const int rc = ad_verify_block(h, drafts, k, nullptr, nullptr, 1);
+  h->profiling = false;
+  g_use_pdl = pdl;
+  cudaEvent_t last = nullptr;
+  if (cudaEventCreate(&last) == cudaSuccess) { cudaEventRecord(last, h->stream); h->prof.emplace_back("end", last); }
+  cudaStreamSynchronize(h->stream);
+  int n = 0;
+  for (size_t i = 0; i + 1 < h->prof.size() && n < capacity; ++i, ++n) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, h->prof[i].second, h->prof[i + 1].second);
+    us[n] = ms * 1e3f;
+    snprintf(names + (size_t)n * 64, 64, "%s", h->prof[i].first.c_str());
+  }
+  for (auto& pr : h->prof) cudaEventDestroy(pr.second);
+  h->prof.clear();
+  *n_launches = n;
+  return rc;
+}
 
 extern "C" int ad_debug_stage_timeline(ad_handle* h, uint64_t* stamps, int32_t capacity, int32_t* n_stages) {
   if (!h || !stamps || !n_stages) return AD_ERR_ARG;

@@ -98,10 +98,18 @@ struct Ctl {
   int ok_flag;
   int M, Mv;
   float mu[NT_MAX], rs[NT_MAX];
+  __align__(16) float gain[1024];   // LayerNorm gain / bias of the columns this CTA stages in the current stage
+  __align__(16) float beta[1024];
   int tok[NT_MAX], pos[NT_MAX], slot[NT_MAX], vrow[NT_MAX];
   float red_val[4][NT_MAX];
   int red_idx[4][NT_MAX];
 };
+
+#ifdef AD_MEGA_DEBUG
+#define MEGA_STAMP(k) do { if (tid == 0 && g == 0 && s < 64) reinterpret_cast<long long*>(p.dbg + 4096)[s * 8 + (k)] = clock64(); } while (0)
+#else
+#define MEGA_STAMP(k) do { } while (0)
+#endif
 
 // ---- small PTX helpers -------------------------------------------------------------------------------------
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
@@ -188,63 +196,101 @@ struct ActSrc {
   int ld;
 };
 
-// Eight consecutive columns (col .. col + 7) of the activation of packed token `row` (metadata index mi), as floats.
-__device__ __forceinline__ void act8(const Params& p, const Ctl* ctl, const ActSrc& a, int row, int col, float* out) {
+// Raw inputs of eight consecutive activation columns of one packed token: loaded first (so that several chunks'
+// loads are in flight at once), turned into values afterwards.
+struct Raw8 {
+  float4 a0, a1;   // SRC_LAZY_LN: x;  SRC_EMBED: positional table
+  uint4 u;         // SRC_PLAIN: the values;  SRC_EMBED: embedding row
+};
+__device__ __forceinline__ void raw8_load(const Params& p, const Ctl* ctl, const ActSrc& a, int row, int col, Raw8& r) {
   if (a.mode == SRC_PLAIN) {
-    unpack8(__ldcg(reinterpret_cast<const uint4*>(a.plain + (size_t)row * a.ld + col)), out);
+    r.u = __ldcg(reinterpret_cast<const uint4*>(a.plain + (size_t)row * a.ld + col));
   } else if (a.mode == SRC_LAZY_LN) {
     const float* xr = a.x + (size_t)row * a.ld + col;
-    const float4 x0 = __ldcg(reinterpret_cast<const float4*>(xr)), x1 = __ldcg(reinterpret_cast<const float4*>(xr + 4));
-    const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.g + col)), g1 = __ldg(reinterpret_cast<const float4*>(a.g + col + 4));
-    const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.b + col)), b1 = __ldg(reinterpret_cast<const float4*>(a.b + col + 4));
+    r.a0 = __ldcg(reinterpret_cast<const float4*>(xr));
+    r.a1 = __ldcg(reinterpret_cast<const float4*>(xr + 4));
+  } else {
+    r.u = __ldg(reinterpret_cast<const uint4*>(p.emb + (size_t)ctl->tok[row] * p.d + col));
+    const float* pr = p.pe + (size_t)ctl->pos[row] * p.d + col;
+    r.a0 = __ldg(reinterpret_cast<const float4*>(pr));
+    r.a1 = __ldg(reinterpret_cast<const float4*>(pr + 4));
+  }
+}
+// gcol: index of `col` inside the gain / bias slice held in shared memory (ctl->gain, ctl->beta)
+__device__ __forceinline__ uint4 raw8_finish(const Params& p, const Ctl* ctl, const ActSrc& a, int row, int gcol, const Raw8& r) {
+  if (a.mode == SRC_PLAIN) return r.u;
+  float o[8];
+  if (a.mode == SRC_LAZY_LN) {
     const float mu = ctl->mu[row], rs = ctl->rs[row];
-    out[0] = g0.x * ((x0.x - mu) * rs) + b0.x; out[1] = g0.y * ((x0.y - mu) * rs) + b0.y;
-    out[2] = g0.z * ((x0.z - mu) * rs) + b0.z; out[3] = g0.w * ((x0.w - mu) * rs) + b0.w;
-    out[4] = g1.x * ((x1.x - mu) * rs) + b1.x; out[5] = g1.y * ((x1.y - mu) * rs) + b1.y;
-    out[6] = g1.z * ((x1.z - mu) * rs) + b1.z; out[7] = g1.w * ((x1.w - mu) * rs) + b1.w;
+    const float4 g0 = *reinterpret_cast<const float4*>(&ctl->gain[gcol]), g1 = *reinterpret_cast<const float4*>(&ctl->gain[gcol + 4]);
+    const float4 b0 = *reinterpret_cast<const float4*>(&ctl->beta[gcol]), b1 = *reinterpret_cast<const float4*>(&ctl->beta[gcol + 4]);
+    o[0] = g0.x * ((r.a0.x - mu) * rs) + b0.x; o[1] = g0.y * ((r.a0.y - mu) * rs) + b0.y;
+    o[2] = g0.z * ((r.a0.z - mu) * rs) + b0.z; o[3] = g0.w * ((r.a0.w - mu) * rs) + b0.w;
+    o[4] = g1.x * ((r.a1.x - mu) * rs) + b1.x; o[5] = g1.y * ((r.a1.y - mu) * rs) + b1.y;
+    o[6] = g1.z * ((r.a1.z - mu) * rs) + b1.z; o[7] = g1.w * ((r.a1.w - mu) * rs) + b1.w;
   } else {
     float e[8];
-    unpack8(__ldg(reinterpret_cast<const uint4*>(p.emb + (size_t)ctl->tok[row] * p.d + col)), e);
-    const float* pr = p.pe + (size_t)ctl->pos[row] * p.d + col;
-    const float4 p0 = __ldg(reinterpret_cast<const float4*>(pr)), p1 = __ldg(reinterpret_cast<const float4*>(pr + 4));
-    out[0] = e[0] * p.emb_scale + p0.x; out[1] = e[1] * p.emb_scale + p0.y;
-    out[2] = e[2] * p.emb_scale + p0.z; out[3] = e[3] * p.emb_scale + p0.w;
-    out[4] = e[4] * p.emb_scale + p1.x; out[5] = e[5] * p.emb_scale + p1.y;
-    out[6] = e[6] * p.emb_scale + p1.z; out[7] = e[7] * p.emb_scale + p1.w;
+    unpack8(r.u, e);
+    o[0] = e[0] * p.emb_scale + r.a0.x; o[1] = e[1] * p.emb_scale + r.a0.y;
+    o[2] = e[2] * p.emb_scale + r.a0.z; o[3] = e[3] * p.emb_scale + r.a0.w;
+    o[4] = e[4] * p.emb_scale + r.a1.x; o[5] = e[5] * p.emb_scale + r.a1.y;
+    o[6] = e[6] * p.emb_scale + r.a1.z; o[7] = e[7] * p.emb_scale + r.a1.w;
   }
-}
-// Four consecutive columns of the same (residual of a sublayer-closing projection).
-__device__ __forceinline__ float4 act4(const Params& p, const Ctl* ctl, const ActSrc& a, int row, int col) {
-  if (a.mode == SRC_LAZY_LN) {
-    const float4 x0 = __ldcg(reinterpret_cast<const float4*>(a.x + (size_t)row * a.ld + col));
-    const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.g + col));
-    const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.b + col));
-    const float mu = ctl->mu[row], rs = ctl->rs[row];
-    return make_float4(g0.x * ((x0.x - mu) * rs) + b0.x, g0.y * ((x0.y - mu) * rs) + b0.y,
-                       g0.z * ((x0.z - mu) * rs) + b0.z, g0.w * ((x0.w - mu) * rs) + b0.w);
-  }
-  const uint2 u = __ldg(reinterpret_cast<const uint2*>(p.emb + (size_t)ctl->tok[row] * p.d + col));
-  const float4 pp = __ldg(reinterpret_cast<const float4*>(p.pe + (size_t)ctl->pos[row] * p.d + col));
-  return make_float4(__uint_as_float(u.x << 16) * p.emb_scale + pp.x, __uint_as_float(u.x & 0xffff0000u) * p.emb_scale + pp.y,
-                     __uint_as_float(u.y << 16) * p.emb_scale + pp.z, __uint_as_float(u.y & 0xffff0000u) * p.emb_scale + pp.w);
+  return pack8(o);
 }
 
-// Per-token mean and reciprocal standard deviation from the partial sums of the producing stage.  Workers only.
-__device__ __forceinline__ void row_stats(const Params& p, Ctl* ctl, const float* stats, int M, int tid) {
-  const int warp = tid >> 5, lane = tid & 31, slabs = p.d >> 7;
-  for (int m = warp; m < M; m += 8) {
+// Residual of a sublayer-closing projection, four consecutive columns: raw loads, then the value.
+struct Raw4 {
+  float4 x, g, b;  // SRC_LAZY_LN: x, gain, bias;  SRC_EMBED: x = positional table
+  uint2 u;         // SRC_EMBED: embedding row
+};
+__device__ __forceinline__ void raw4_load(const Params& p, const Ctl* ctl, const ActSrc& a, int row, int col, Raw4& r) {
+  if (a.mode == SRC_LAZY_LN) {
+    r.x = __ldcg(reinterpret_cast<const float4*>(a.x + (size_t)row * a.ld + col));
+    r.g = __ldg(reinterpret_cast<const float4*>(a.g + col));
+    r.b = __ldg(reinterpret_cast<const float4*>(a.b + col));
+  } else {
+    r.u = __ldg(reinterpret_cast<const uint2*>(p.emb + (size_t)ctl->tok[row] * p.d + col));
+    r.x = __ldg(reinterpret_cast<const float4*>(p.pe + (size_t)ctl->pos[row] * p.d + col));
+  }
+}
+__device__ __forceinline__ float4 raw4_finish(const Params& p, const Ctl* ctl, const ActSrc& a, int row, const Raw4& r) {
+  if (a.mode == SRC_LAZY_LN) {
+    const float mu = ctl->mu[row], rs = ctl->rs[row];
+    return make_float4(r.g.x * ((r.x.x - mu) * rs) + r.b.x, r.g.y * ((r.x.y - mu) * rs) + r.b.y,
+                       r.g.z * ((r.x.z - mu) * rs) + r.b.z, r.g.w * ((r.x.w - mu) * rs) + r.b.w);
+  }
+  return make_float4(__uint_as_float(r.u.x << 16) * p.emb_scale + r.x.x, __uint_as_float(r.u.x & 0xffff0000u) * p.emb_scale + r.x.y,
+                     __uint_as_float(r.u.y << 16) * p.emb_scale + r.x.z, __uint_as_float(r.u.y & 0xffff0000u) * p.emb_scale + r.x.w);
+}
+
+// Per-token mean and reciprocal standard deviation from the partial sums of the producing stage (four threads per
+// token, one round trip for all tokens), and the LayerNorm gain / bias slice [col0, col0 + ncols) into shared memory.
+// Workers only; ends with a worker barrier.  stats == null: only the barrier.
+__device__ __forceinline__ void row_stats(const Params& p, Ctl* ctl, const float* stats, int M, int tid, const float* gain,
+                                          const float* beta, int col0, int ncols) {
+  if (stats) {
+    const int m = tid >> 2, part = tid & 3, slabs = p.d >> 7;
     float s1 = 0.f, s2 = 0.f;
-    if (lane < slabs) {
-      const float2 v = __ldcg(reinterpret_cast<const float2*>(stats + ((size_t)lane * p.M_cap + m) * 2));
-      s1 = v.x; s2 = v.y;
+    if (m < M) {
+      float2 v0 = make_float2(0.f, 0.f), v1 = v0;
+      if (part < slabs) v0 = __ldcg(reinterpret_cast<const float2*>(stats + ((size_t)part * p.M_cap + m) * 2));
+      if (part + 4 < slabs) v1 = __ldcg(reinterpret_cast<const float2*>(stats + ((size_t)(part + 4) * p.M_cap + m) * 2));
+      s1 = v0.x + v1.x; s2 = v0.y + v1.y;
     }
-#pragma unroll
-    for (int o = 4; o > 0; o >>= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s2 += __shfl_xor_sync(0xffffffffu, s2, o); }
-    if (lane == 0) {
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 1); s2 += __shfl_xor_sync(0xffffffffu, s2, 1);
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 2); s2 += __shfl_xor_sync(0xffffffffu, s2, 2);
+    if (part == 0 && m < M) {
       const float mean = s1 / (float)p.d;
       const float var = fmaxf(s2 / (float)p.d - mean * mean, 0.f);
       ctl->mu[m] = mean;
       ctl->rs[m] = rsqrtf(var + p.eps);
+    }
+    if (gain) {
+      for (int i = tid; i < (ncols >> 2); i += N_WORKERS) {
+        *reinterpret_cast<float4*>(&ctl->gain[i * 4]) = __ldg(reinterpret_cast<const float4*>(gain + col0 + i * 4));
+        *reinterpret_cast<float4*>(&ctl->beta[i * 4]) = __ldg(reinterpret_cast<const float4*>(beta + col0 + i * 4));
+      }
     }
   }
   worker_sync();
@@ -254,21 +300,38 @@ __device__ __forceinline__ void row_stats(const Params& p, Ctl* ctl, const float
 // 128-byte-swizzled K-major layout the MMA descriptor expects (16-byte chunk c of row r at chunk c ^ (r & 7)).
 // rows: packed row of each tile row (null: identity); rows >= n_valid are zero.  yb_out != null: the staged values
 // are also written there as plain rows (the normalised hidden states, for the debug paths).
-__device__ __forceinline__ void stage_b(const Params& p, const Ctl* ctl, const ActSrc& a, int kb0, int n_kb, int ntile,
-                                        int n_valid, const int* rows, uint32_t b_smem, bf16* yb_out, int tid) {
-  const int per_kb = ntile * 8;
-  for (int idx = tid; idx < n_kb * per_kb; idx += N_WORKERS) {
-    const int kbl = idx / per_kb, rem = idx - kbl * per_kb;
-    const int m = rem >> 3, c = rem & 7;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (m < n_valid) {
-      float f[8];
-      const int row = rows ? rows[m] : m;
-      act8(p, ctl, a, row, (kb0 + kbl) * 64 + c * 8, f);
-      v = pack8(f);
-      if (yb_out) *reinterpret_cast<uint4*>(yb_out + (size_t)m * a.ld + (kb0 + kbl) * 64 + c * 8) = v;
+// The raw loads of the first batch of chunks are issued BEFORE the row statistics are fetched, so that both round
+// trips overlap; stats / gain / beta as for row_stats (all null when nothing is normalised here or later in the stage).
+constexpr int STAGE_NB = 4;      // 16-byte chunks a thread has in flight
+__device__ __forceinline__ void stage_b(const Params& p, Ctl* ctl, const ActSrc& a, int kb0, int n_kb, int ntile,
+                                        int n_valid, const int* rows, uint32_t b_smem, bf16* yb_out, int tid,
+                                        const float* stats, int M, const float* gain, const float* beta) {
+  const int per_kb = ntile * 8, total = n_kb * per_kb;
+  const int n_batches = (total + N_WORKERS * STAGE_NB - 1) / (N_WORKERS * STAGE_NB);
+  for (int bt = 0; bt < n_batches; ++bt) {
+    Raw8 raw[STAGE_NB];
+#pragma unroll
+    for (int i = 0; i < STAGE_NB; ++i) {
+      const int idx = (bt * STAGE_NB + i) * N_WORKERS + tid;
+      if (idx < total) {
+        const int kbl = idx / per_kb, rem = idx - kbl * per_kb, m = rem >> 3, c = rem & 7;
+        if (m < n_valid) raw8_load(p, ctl, a, rows ? rows[m] : m, (kb0 + kbl) * 64 + c * 8, raw[i]);
+      }
     }
-    st_shared_u4(b_smem + (uint32_t)(kbl * ntile * 128 + m * 128 + ((c ^ (m & 7)) << 4)), v);
+    if (bt == 0) row_stats(p, ctl, stats, M, tid, gain, beta, kb0 * 64, n_kb * 64);
+#pragma unroll
+    for (int i = 0; i < STAGE_NB; ++i) {
+      const int idx = (bt * STAGE_NB + i) * N_WORKERS + tid;
+      if (idx < total) {
+        const int kbl = idx / per_kb, rem = idx - kbl * per_kb, m = rem >> 3, c = rem & 7;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (m < n_valid) {
+          v = raw8_finish(p, ctl, a, rows ? rows[m] : m, kbl * 64 + c * 8, raw[i]);
+          if (yb_out) *reinterpret_cast<uint4*>(yb_out + (size_t)m * a.ld + (kb0 + kbl) * 64 + c * 8) = v;
+        }
+        st_shared_u4(b_smem + (uint32_t)(kbl * ntile * 128 + m * 128 + ((c ^ (m & 7)) << 4)), v);
+      }
+    }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA's reads
 }
@@ -554,6 +617,7 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
           if (!ok) break;
         }
         if (p.timeline && g == 0 && tid == 0) p.timeline[2 * s] = gs::now_ns();
+        MEGA_STAMP(0);
         // the x / statistics buffer holding this layer's input, and the other one
         const int in_buf = si.layer & 1, oth = in_buf ^ 1;
 
@@ -608,11 +672,13 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
               lazy(bsrc, L & 1, p.layers[L - 1].ln3g, p.layers[L - 1].ln3b);
               break;
           }
-          if (stats_in) row_stats(p, ctl, stats_in, M, tid);
+          // LayerNorm gain / bias of the staged operand (null when the operand is not normalised here)
+          const float* bg = bsrc.mode == SRC_LAZY_LN ? bsrc.g : nullptr;
+          const float* bb = bsrc.mode == SRC_LAZY_LN ? bsrc.b : nullptr;
 
           if (vocab) {
             // B operand resident for the whole stage; tiles g, g + G, ...; epilogue of tile i under the MMAs of tile i + 1
-            stage_b(p, ctl, bsrc, 0, si.K >> 6, ntile, Mv, ctl->vrow, b_base, g == 0 ? p.yb_out : nullptr, tid);
+            stage_b(p, ctl, bsrc, 0, si.K >> 6, ntile, Mv, ctl->vrow, b_base, g == 0 ? p.yb_out : nullptr, tid, stats_in, M, bg, bb);
             __syncwarp();
             if (lane == 0) mbar_arrive_local(tc::smem_u32(&ctl->b_ready));
             for (int nt = g; nt < n_tiles; nt += G) {
@@ -655,23 +721,14 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
             const int tpc = ntile / CS;                      // tokens this CTA reduces and finishes
             for (int nt = c; nt < n_tiles; nt += NC) {
               const uint32_t a = jc & 1, pb = rc & 1;
-              stage_b(p, ctl, bsrc, r * kpc, kpc, ntile, M, nullptr, b_base, nullptr, tid);
-#ifdef AD_MEGA_DEBUG
-              worker_sync();
-              if (tid == 0 && g < 16 && s < 32) {
-                float sb = 0.f;
-                const unsigned short* bp = reinterpret_cast<const unsigned short*>(flex_ptr);
-                for (int i = 0; i < kpc * ntile * 64; ++i) sb += fabsf(__uint_as_float((uint32_t)bp[i] << 16));
-                p.dbg[(g * 32 + s) * 4 + 0] = sb;
-                p.dbg[(g * 32 + s) * 4 + 2] = (float)jc;
-                p.dbg[(g * 32 + s) * 4 + 3] = (float)rc;
-              }
-              worker_sync();
-#endif
+              // (the statistics are the same for every tile of the stage: fetched with the first one)
+              stage_b(p, ctl, bsrc, r * kpc, kpc, ntile, M, nullptr, b_base, nullptr, tid, nt == c ? stats_in : nullptr, M, bg, bb);
               __syncwarp();
               if (lane == 0) mbar_arrive_local(tc::smem_u32(&ctl->b_ready));
+              MEGA_STAMP(1);
               ok = worker_all(wait_bar(tc::smem_u32(&ctl->acc_full[a]), (jc >> 1) & 1, ctl, p.status));
               if (!ok) break;
+              MEGA_STAMP(2);
               asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
               // this CTA's partial [tokens x 128 features] -> reduction buffer pb
               float* red = red_ptr + (size_t)pb * (p.red_bytes / 4);
@@ -686,34 +743,32 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
               __syncwarp();
               if (lane == 0) mbar_arrive_local(tc::smem_u32(&ctl->acc_empty[a]));
               worker_sync();                                 // the whole partial is in shared memory
-#ifdef AD_MEGA_DEBUG
-              if (tid == 0 && g < 16 && s < 32) {
-                float sr = 0.f;
-                for (int i = 0; i < ntile * RED_LD; ++i) sr += fabsf(red[i]);
-                p.dbg[(g * 32 + s) * 4 + 1] = sr;
-              }
-#endif
+              MEGA_STAMP(3);
               if (tid < CS) mbar_arrive_remote(tc::smem_u32(&ctl->red_full[pb]), (uint32_t)tid);
               ok = worker_all(wait_bar(tc::smem_u32(&ctl->red_full[pb]), (rc >> 1) & 1, ctl, p.status, true));
               if (!ok) break;
+              MEGA_STAMP(4);
               // sum the CS partials of this CTA's tokens in rank order; lane owns features 4 lane .. 4 lane + 3
               for (int tl_ = warp; tl_ < tpc; tl_ += 8) {
                 const int m = r * tpc + tl_;
                 if (m >= M) continue;
                 const uint32_t local = red_base + (uint32_t)pb * (uint32_t)p.red_bytes + (uint32_t)((m * RED_LD + lane * 4) * 4);
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int q = 0; q < CS; ++q) {
-                  const float4 o = ld_dsmem_f4(map_to_rank(local, (uint32_t)q));
-#ifdef AD_MEGA_DEBUG
-                  if (tid == 0 && g < 16 && s < 16 && q < 4) p.dbg[(g * 32 + s + 16) * 4 + q] = o.x;
-#endif
-                  v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                }
                 const int n = nt * 128 + lane * 4;
+                // all loads first: the CS partials, the bias and the residual's inputs are one round trip together
+                float4 part[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  if (q < CS) part[q] = ld_dsmem_f4(map_to_rank(local, (uint32_t)q));
                 const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + n));
+                Raw4 rr;
+                if (x_out) raw4_load(p, ctl, rsrc, m, n, rr);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  if (q < CS) { v.x += part[q].x; v.y += part[q].y; v.z += part[q].z; v.w += part[q].w; }
                 v.x += bv.x; v.y += bv.y; v.z += bv.z; v.w += bv.w;
                 if (x_out) {
-                  const float4 rv = act4(p, ctl, rsrc, m, n);
+                  const float4 rv = raw4_finish(p, ctl, rsrc, m, rr);
                   v.x += rv.x; v.y += rv.y; v.z += rv.z; v.w += rv.w;
                   *reinterpret_cast<float4*>(x_out + (size_t)m * p.d + n) = v;
                   float s1 = v.x + v.y + v.z + v.w, s2 = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -736,6 +791,7 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
                   *reinterpret_cast<uint2*>(dst) = u;
                 }
               }
+              MEGA_STAMP(5);
               worker_sync();
               ++jc; ++rc;
             }
@@ -749,8 +805,12 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
       __threadfence();
 #endif
       worker_sync();
+      MEGA_STAMP(6);
       if (tid == 0) {
         gs::arrive_release(p.sync_ctr + (size_t)s * SYNC_STRIDE, 1u);
+#ifdef AD_MEGA_DEBUG
+        if (g == 0 && s < 64) reinterpret_cast<long long*>(p.dbg + 4096)[s * 8 + 7] = clock64();
+#endif
         if (p.timeline && g == 0) p.timeline[2 * s + 1] = gs::now_ns();
       }
     }

@@ -733,6 +733,42 @@ __global__ void export_block_kernel(DevState st, Dims dm, int* argmax_out, int* 
   }
 }
 
+// End of ad_generate: everything the host needs, gathered into one block (device pointer of pinned, mapped host memory
+// or a device buffer), so that the call ends with ONE synchronisation and no further copies:
+//   block[0] = iterations the device-side loop ran, block[1] = latched status word (cleared here),
+//   block[2] = iterations with an active row, block[3] = B,
+//   block[4 + 4 b ..] = {row iterations, accepted, offered, output length} of row b,
+//   block[4 + 4 B + b * max_tgt ..] = output ids of row b (only when out_dev is null: host-resident results).
+// out_dev / out_len_dev (device pointers, may be null): the caller's result arrays when they live on the device.
+// grid = B, block = 128.
+__global__ void __launch_bounds__(128)
+finalize_generate_kernel(DevState st, Dims dm, int* out_dev, int out_stride, int* out_len_dev, int* block) {
+  pdl_launch();
+  pdl_wait();
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int len = st.len[b];
+  if (tid == 0) {
+    if (b == 0) {
+      block[0] = st.loop_it[2];
+      block[1] = *st.status;
+      *st.status = 0;
+      block[2] = st.loop_it[0];
+      block[3] = dm.B;
+    }
+    int* row = block + 4 + 4 * b;
+    row[0] = st.stat_it[b]; row[1] = st.stat_acc[b]; row[2] = st.stat_off[b]; row[3] = len;
+    if (out_len_dev) out_len_dev[b] = len;
+  }
+  const int* src = st.out_ids + (size_t)b * dm.max_tgt;
+  if (out_dev) {
+    const int w = min(out_stride, dm.max_tgt);
+    for (int i = tid; i < w; i += 128) out_dev[(size_t)b * out_stride + i] = src[i];
+  } else {
+    int* dst = block + 4 + 4 * dm.B + (size_t)b * dm.max_tgt;
+    for (int i = tid; i < dm.max_tgt; i += 128) dst[i] = src[i];
+  }
+}
+
 // FP32 copy of an activation buffer (debug).  grid-stride.
 template <typename ActT>
 __global__ void to_f32_kernel(const ActT* __restrict__ src, float* __restrict__ dst, size_t n) {
