@@ -483,3 +483,131 @@ def run_ours(args, rank, world, local_rank):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def bench_extras(args, binding, dec, w, dev, pk, flush, t_src, t_len, t_max, t_out, t_olen, value, world):
+    """Everything beside the headline: per-kernel table, fixed-shape steps, tensor regime, greedy baseline, the other
+    workload recipes.  Rank 0 only; each part is bounded so that the default run stays within a few minutes."""
+    import torch
+    extras = {}
+    shape = synth.BASE
+    V, d = shape.vocab, shape.d_model
+    wv = weight_bytes(shape)
+
+    # every kernel of one step on its own (block of 40 tokens, empty prefix, first sentence's source)
+    dec.encode(t_src[:1].cpu().numpy(), t_len[:1].cpu().numpy())
+    drafts = np.random.default_rng(3).integers(4, V, size=(1, KMAX)).astype(np.int32)
+    extras["kernels"] = kernel_table(dec, shape, drafts, KMAX, pk)
+
+    # the projection + arg-max kernel alone (the largest kernel by bytes): one launch between two events
+    lib = dec.lib
+    M = KMAX
+    x = torch.randn((M, d), device=dev).bfloat16()
+    emb = dec._keep[0][: V * d].view(V, d)
+    nb = lib.ad_vocab_argmax_scratch_bytes(V, M)
+    scratch = torch.empty(nb + 256, dtype=torch.uint8, device=dev)
+    sbase = (scratch.data_ptr() + 255) // 256 * 256
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def vocab_once():
+        assert lib.ad_vocab_argmax(C.c_void_p(x.data_ptr()), C.c_void_p(emb.data_ptr()), 1, M, d, V, None, C.c_void_p(sbase), nb,
+                                   C.c_void_p(status.data_ptr()), C.c_void_p(dec.stream.cuda_stream)) == 0
+    vb = V * d * 2 + M * d * 2 + M * 4
+    t_cold = statistics.mean(_events(dec.stream, vocab_once, 20, flush))
+    t_warm = statistics.mean(_events(dec.stream, vocab_once, 20))
+    extras["projection_kernel"] = dict(kernel="gemm_tc_kernel<EPI_ARGMAX>, vocabulary 32000 x 512, 40 tokens", algorithmic_bytes=vb,
+                                       us_cold=t_cold, us_l2_warm=t_warm, gbs_cold=vb / (t_cold * 1e-6) / 1e9,
+                                       frac_of_hbm_peak_cold=vb / (t_cold * 1e-6) / 1e9 / pk["hbm_gbs"],
+                                       traffic_ncu=32855040, traffic_note="dram__bytes_read.sum + dram__bytes_write.sum of one launch "
+                                       "(profiles/vocab_argmax_gemm_base_M40_ncu_full.txt; this kernel is unchanged since that capture)")
+
+    # fixed-shape verification steps, weight-streaming regime (direct launches): L2-warm and L2-flushed
+    pts = []
+    for (k, prefix) in ((16, 16), (64, 0), (1, 20)):
+        warm, cold = fixed_step(binding, shape, w, pk, 1, k, prefix, 32, reps=30, flush=flush)
+        bts = step_bytes(shape, 32, prefix + k, k)
+        pts.append(dict(shape=f"base, batch 1, block {k} on a {prefix}-token prefix, source 32", algorithmic_bytes=bts,
+                        us_l2_warm=warm, us_l2_flushed=cold, hbm_floor_us=bts / (pk["hbm_gbs"] * 1e9) * 1e6,
+                        frac_l2_warm=bts / (warm * 1e-6) / 1e9 / pk["hbm_gbs"], frac_l2_flushed=bts / (cold * 1e-6) / 1e9 / pk["hbm_gbs"]))
+    extras["step_points"] = dict(note="direct launches (no graph), verify + discard; flushed = 256 MB write before every step", points=pts)
+
+    # the library's own greedy decoding (block size 1) of the same sentences
+    def step_greedy():
+        acc = 0
+        for s in range(N_SENT):
+            st = dec.generate_device(t_src[s: s + 1], t_len[s: s + 1], t_out[s: s + 1], t_olen[s: s + 1], mode="IAD", k=1,
+                                     max_len_t=t_max[s: s + 1])
+            acc += st["accepted"]
+        return acc
+    step_greedy()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(dec.stream); g_tok = step_greedy(); g1.record(dec.stream)
+    dec.stream.synchronize()
+    greedy_tps = g_tok / (g0.elapsed_time(g1) * 1e-3)
+    extras["greedy"] = dict(value=greedy_tps, unit=UNIT, speedup_of_draft_verify=value / world / greedy_tps if greedy_tps > 0 else None,
+                            note="same sentences decoded with block size 1 (one token per iteration), encoder included, one pass")
+
+    # tensor-core regime: one verification step of 32 rows x 64 block positions (2048 packed tokens)
+    B32, K32, S32 = 32, 64, 64
+    us32, _ = fixed_step(binding, shape, w, pk, B32, K32, 0, S32, reps=10)
+    M32 = B32 * K32
+    flops32 = 2.0 * (wv / 2) * M32 + 4.0 * 6 * d * (B32 * sum(i + 1 + S32 for i in range(K32)))
+    extras["tensor_regime"] = dict(us_per_step=us32, packed_tokens=M32, flops=flops32, tflops=flops32 / (us32 * 1e-6) / 1e12,
+                                   peak_tflops_burst=pk["bf16_tflops"], peak_tflops_sustained=pk["bf16_tflops_sustained"],
+                                   tensor_floor_us=flops32 / (pk["bf16_tflops"] * 1e12) * 1e6,
+                                   frac_of_floor=flops32 / (pk["bf16_tflops"] * 1e12) * 1e6 / us32,
+                                   frac_of_sustained=flops32 / (pk["bf16_tflops_sustained"] * 1e12) * 1e6 / us32,
+                                   note="batch 32, block 64, empty prefix, source 64; direct launches, weights L2-warm")
+
+    # the other workload recipes (and shapes) through ad_generate, the CPU checker's bounded sample beside each
+    if not args.skip_workloads:
+        oc = args.cpu_seconds / 3 if world == 1 else 0.0
+        wls = [run_workload(binding, 3, w, None, dev, 1, oc, pk)]
+        wn = synth.make_weights(shape, 1)
+        wls.append(run_workload(binding, 5, w, wn, dev, 1, oc, pk))
+        del wn
+        wb, wbn = synth.make_weights(synth.BIG, 0), synth.make_weights(synth.BIG, 1)
+        wls.append(run_workload(binding, 4, wb, wbn, dev, 4, oc, pk))
+        del wb, wbn
+        extras["workloads"] = wls
+        shp = []
+        for sh, k in ((synth.DEEP_ENC, 40), (synth.BART_BASE_SIZED, 25)):
+            ws = synth.make_weights(sh, 0)
+            warm, cold = fixed_step(binding, sh, ws, pk, 1, k, 0, 32, reps=20, flush=flush)
+            bts = step_bytes(sh, 32, k, k)
+            shp.append(dict(shape=f"{sh.name} ({sh.n_enc}+{sh.n_dec}, d{sh.d_model}, vocab {sh.vocab}), batch 1, block {k}, source 32",
+                            algorithmic_bytes=bts, us_l2_warm=warm, us_l2_flushed=cold,
+                            frac_l2_warm=bts / (warm * 1e-6) / 1e9 / pk["hbm_gbs"]))
+            del ws
+        extras["other_shapes"] = shp
+        if world == 1:      # the checker on ONE thread, once (the same sample as cpu_baseline, a third of its time budget)
+            from oracle import ad_oracle as O
+            n0 = O.threads()
+            O.set_threads(1)
+            one, _, _, _ = oracle_sample(args.cpu_seconds / 3)
+            O.set_threads(n0)
+            extras["cpu_baseline_1_thread"] = one
+    return extras
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sync-every", type=int, default=0, help="iterations between host checks of the finished flag (0 = library default)")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work of the checker baseline sample")
+    ap.add_argument("--skip-workloads", action="store_true", help="leave out the other workload recipes and shapes")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
