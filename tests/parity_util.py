@@ -49,11 +49,22 @@ def check_block(gpu_ids, gpu_n, drafts, res, k, eos, where=""):
     return stats
 
 
-def lockstep(dec, model, src, lens, streams, kcap, max_lens, tol, max_steps=None, check_logits=True):
+def lockstep(dec, model, src, lens, streams, kcap, max_lens, tol, max_steps=None, check_logits=True, check_rows=None,
+             states=None):
     """Walks a batch through draft-verify along the checker's trajectory.  streams[b] is the position-aligned
-    draft stream of row b.  Returns summary statistics."""
+    draft stream of row b.  check_rows: the rows compared with the checker (default: all); the other rows run in the
+    same batch along the library's own trajectory (their own predictions are committed), which keeps the CPU cost of
+    a wide batch bounded while every checked row still shares its passes with all the others.
+    states: checker states of the rows to reuse (their encoder pass is then not repeated); they are reset here.
+    Returns summary statistics."""
     B = len(lens)
-    states = [model.state(src[b, : lens[b]], cap=dec.max_tgt) for b in range(B)]
+    checked = set(range(B)) if check_rows is None else set(check_rows)
+    if states is None:
+        states = [model.state(src[b, : lens[b]], cap=dec.max_tgt) if b in checked else None for b in range(B)]
+    for st in states:
+        if st is not None:
+            st.reset()
+    own_len = [0] * B
     dec.encode(src, lens)
     last = [model.bos] * B
     fin = [False] * B
@@ -66,7 +77,7 @@ def lockstep(dec, model, src, lens, streams, kcap, max_lens, tol, max_steps=None
         for b in range(B):
             if fin[b]:
                 continue
-            ln = states[b].len
+            ln = states[b].len if b in checked else own_len[b]
             ks[b] = min(kcap, int(max_lens[b]) - ln)
             seg = np.asarray(streams[b][ln: ln + ks[b]], np.int32)
             drafts[b, : len(seg)] = seg
@@ -80,6 +91,17 @@ def lockstep(dec, model, src, lens, streams, kcap, max_lens, tol, max_steps=None
             k = int(ks[b])
             if k == 0:
                 assert gpu_n[b] == 0
+                continue
+            if b not in checked:          # the library's own trajectory
+                n = int(gpu_n[b])
+                assert 1 <= n <= k
+                tokens[b, :n] = gpu_ids[b, :n]
+                ns[b] = n
+                own_len[b] += n
+                last[b] = int(gpu_ids[b, n - 1])
+                fin[b] = last[b] == model.eos or own_len[b] >= int(max_lens[b])
+                lib_fin[b] = last[b] == model.eos or own_len[b] >= dec.max_tgt
+                off += k
                 continue
             res = states[b].verify_block(last[b], drafts[b, :k], want_logits=True)
             if check_logits:
@@ -101,7 +123,8 @@ def lockstep(dec, model, src, lens, streams, kcap, max_lens, tol, max_steps=None
         dec.force_commit(tokens, ns)
         ln, lt, fn = dec.state()
         for b in range(B):
-            assert ln[b] == states[b].len, f"cache length of row {b}: {ln[b]} != {states[b].len}"
+            want = states[b].len if b in checked else own_len[b]
+            assert ln[b] == want, f"cache length of row {b}: {ln[b]} != {want}"
             assert lt[b] == last[b]
             assert bool(fn[b]) == lib_fin[b]
         step += 1

@@ -210,6 +210,12 @@ def test_workload3_base_batch32(base_weights):
     greedy, streams = _greedy_streams(om, src, lens, max_len, wl.agreement, wl.index, wl.shape.vocab)
     tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, max_steps=2)
     assert tot["steps"] == 2
+    print(f"recipe 3, two iterations, all 32 rows: {tot}")
+    # four rows to the END of their sentences in lock-step with the checker while all 32 rows run (the other 28 follow the
+    # library's own trajectory): per-row accepted lengths and cache commits stay independent in a wide ragged batch
+    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, check_rows=[0, 5, 17, 31])
+    assert tot["tokens"] == sum(len(greedy[b][0]) for b in (0, 5, 17, 31))
+    print(f"recipe 3, rows 0/5/17/31 to completion: {tot}")
     outs, stats = dec.generate(src, lens, mode="IAD", k=wl.k, max_len=max_len, draft_override=streams)
     for b in range(wl.batch):
         P.check_free_run(outs[b], greedy[b][0], greedy[b][1], f"row {b}")
@@ -238,8 +244,9 @@ def test_workload4_big_generalized():
     _drafter_parity(dec, on, src, lens, wl.k)
     st = P.drafter_at_prefix(dec, on, src, lens, [greedy[0][0][:9]], wl.k, TOL_BF16)
     print(f"big drafter at a 9-token prefix: {st}")
-    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16, max_steps=3)
-    assert tot["steps"] >= 1
+    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, max_len, TOL_BF16)     # the whole sentence
+    assert tot["tokens"] == len(greedy[0][0])
+    print(f"recipe 4, one sentence to completion: {tot}")
     outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=max_len, draft_override=streams, run_drafter=True)
     P.check_free_run(outs[0], greedy[0][0], greedy[0][1], "big")
 
@@ -252,28 +259,32 @@ def test_workload5_base_long_source_batch8(base_weights):
     on = O.Model(synth.BASE, wn, max_pos=401)
     src, lens = synth.make_sources(wl)
     max_len = synth.max_out_lens(wl, lens)
-    # a perfect stream is not needed for lock-step: take uniform random drafts mixed with the checker's own
-    # first greedy tokens so that several positions are accepted
-    states = [om.state(src[b, : lens[b]], cap=80) for b in range(2)]
+    # All 8 rows in lock-step with the checker for 12 iterations at agreement 0.6 (about 2.5 tokens accepted per row and
+    # iteration): every iteration rolls the rejected part of a 25-token block back, and the cache is some 25 positions
+    # deep by the end.  The checker pays the 400-token encoder once per row.
+    T = 40
+    states = [om.state(src[b, : lens[b]], cap=80) for b in range(8)]
     dec.encode(src, lens)
     mem = dec.debug_encoder_memory(1, int(lens[1]))
     assert np.abs(mem - states[1].memory()).max() < TOL_BF16
     _drafter_parity(dec, on, src[:1], lens[:1], 5)
-    g8 = [st.greedy(8) for st in states]
-    streams = np.full((8, 80), 7, np.int32)
-    for b in range(2):
-        streams[b, : len(g8[b][0])] = g8[b][0]
-        streams[b, 5] = 9
-    # only rows 0 and 1 are checked against the checker (the others run but would cost minutes on the CPU)
-    dec2_src, dec2_lens = src[:2], lens[:2]
-    tot = P.lockstep(dec, om, dec2_src, dec2_lens, list(streams[:2]), wl.k, [80, 80], TOL_BF16, max_steps=2)
-    assert tot["steps"] == 2
-    # full batch, free running, repeated rollbacks (agreement 0.6 on a random stream): the loop must terminate
-    outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=np.full(8, 12, np.int32), draft_override=streams,
+    gT = [st.greedy(T) for st in states]
+    g = np.full((8, 80), synth.PAD, np.int32)
+    gl = np.zeros(8, np.int32)
+    for b in range(8):
+        g[b, : len(gT[b][0])] = gT[b][0]; gl[b] = len(gT[b][0])
+    streams = synth.corrupt_stream(g, gl, wl.agreement, wl.shape.vocab, wl.index)
+    tot = P.lockstep(dec, om, src, lens, list(streams), wl.k, np.full(8, T), TOL_BF16, max_steps=12, states=states)
+    assert tot["steps"] == 12 or tot["tokens"] == int(gl.sum())
+    ln, _, _ = dec.state()
+    print(f"recipe 5, 8 rows x {tot['steps']} iterations, cache depths {list(ln)}: {tot}")
+    assert max(ln) >= 20
+    # full batch, free running with the drafter: the loop must terminate and agree with the checker's greedy output
+    outs, stats = dec.generate(src, lens, mode="GAD", k=wl.k, max_len=np.full(8, T, np.int32), draft_override=streams,
                                run_drafter=True)
-    assert all(1 <= len(o) <= 12 for o in outs)
-    for b in range(2):
-        P.check_free_run(outs[b][:8], g8[b][0][:len(outs[b][:8])], g8[b][1], f"row {b}")
+    assert all(1 <= len(o) <= T for o in outs)
+    for b in range(8):
+        P.check_free_run(outs[b], gT[b][0], gT[b][1], f"row {b}")
 
 
 def test_long_source_short_blocks(base_weights):
