@@ -330,6 +330,29 @@ def test_deep_encoder_shallow_decoder_shape():
     dec.close()
 
 
+def test_twelve_plus_two_model_at_its_real_shape():
+    """The 12-layer-encoder / 2-layer-decoder model of Section 4.1.2 at its real width (d_model 512, 8 heads, FFN 2048,
+    vocabulary 32000): encoder memory after twelve layers, two lock-step verification steps and the free run."""
+    shape = synth.DEEP_ENC
+    dec, om, _ = make(shape, 1, 24, 24, 24)
+    r = np.random.default_rng(41)
+    src = r.integers(4, shape.vocab, size=(1, 24)).astype(np.int32)
+    lens = np.array([20], np.int32)
+    src[0, 20:] = synth.PAD
+    st = om.state(src[0, :20])
+    g, margin = st.greedy(20)
+    stream = synth.corrupt_stream(g[None, :], [len(g)], 0.85, shape.vocab, 41)[0]
+    dec.encode(src, lens)
+    mem = dec.debug_encoder_memory(0, 20)
+    assert np.abs(mem - st.memory()).max() < 5e-2
+    tot = P.lockstep(dec, om, src, lens, [stream], 24, [20], TOL_BF16, max_steps=2)
+    assert tot["steps"] == 2 and tot["worst_logit_err"] < TOL_BF16
+    print(f"12+2 model: {tot}")
+    outs, _ = dec.generate(src, lens, mode="IAD", k=24, max_len=[20], draft_override=stream[None, :])
+    P.check_free_run(outs[0], g, margin, "12+2")
+    dec.close()
+
+
 def test_bart_base_sized_shape_two_steps():
     """d_model 768, 12 heads, FFN 3072, vocabulary 50265 (393 projection tiles, the last one ragged), the size of the
     models of Section 4.2.4: encoder memory and two lock-step verification steps of a 10-token block."""
