@@ -152,9 +152,6 @@ struct ad_handle {
   mega::LayerPtrs* mega_layers[2] = {nullptr, nullptr};    // [0] verification pass, [1] drafter pass
   float* mega_stats[2] = {nullptr, nullptr};
   unsigned long long* mega_timeline = nullptr;
-#ifdef AD_MEGA_DEBUG
-  float* mega_dbg = nullptr;
-#endif
   unsigned long long cond_handle = 0;   // non-zero only while the body of a device-side `while` node is captured
 };
 
@@ -328,9 +325,6 @@ size_t layout(ad_handle* h, void* base) {
     h->mega_stats[i] = (float*)bp.take(sizeof(float) * 2 * (size_t)(d / 128 + 1) * M_all);
   }
   h->mega_timeline = (unsigned long long*)bp.take(sizeof(unsigned long long) * 2 * (size_t)(mega::ST_PER_LAYER * c.n_dec + 1));
-#ifdef AD_MEGA_DEBUG
-  h->mega_dbg = (float*)bp.take(sizeof(float) * 4096 + 8 * 64 * 8);
-#endif
   for (int k = 0; k < PK_COUNT; ++k) plan_take(bp, h->pass[k].plan, B, h->pass[k].M_cap);
   DevState& s = h->st;
   auto ints = [&](size_t n) { return (int*)bp.take(sizeof(int) * n, 256); };
@@ -776,10 +770,6 @@ int mega_launch(ad_handle* h, int pk) {
   p.B = h->dims.B;
   static const bool trace = [] { const char* e = getenv("AD_MEGA_TIMELINE"); return e && e[0] == '1'; }();
   p.timeline = trace ? h->mega_timeline : nullptr;
-#ifdef AD_MEGA_DEBUG
-  { const char* e = getenv("AD_MEGA_STOP"); p.debug_stop = e ? atoi(e) : 1 << 20; }
-  p.dbg = h->mega_dbg;
-#endif
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(h->mega_cs * h->mega_nc); cfg.blockDim = dim3(mega::THREADS);
   cfg.dynamicSmemBytes = h->mega_smem; cfg.stream = h->stream;
@@ -1495,30 +1485,6 @@ extern "C" int ad_debug_encoder_memory(ad_handle* h, int32_t b, float* mem, size
   return AD_OK;
 }
 
-#ifdef AD_MEGA_DEBUG
-// Debugging builds only: raw copy of an internal buffer (0/1: x, 2/3: statistics, 4: q, 5: attention output, 6: FFN hidden,
-// 7: yb, 8/9: self-attention keys / values of layer `layer`).
-extern "C" int ad_debug_peek(ad_handle* h, int which, int layer, void* dst, size_t bytes) {
-  const size_t self_layer = (size_t)h->cfg.max_tgt * h->cfg.max_batch * h->cfg.d_model * h->esz;
-  const void* src = nullptr;
-  switch (which) {
-    case 0: src = h->y; break;
-    case 1: src = h->pre; break;
-    case 2: src = h->mega_stats[0]; break;
-    case 3: src = h->mega_stats[1]; break;
-    case 4: src = h->qbuf; break;
-    case 5: src = h->abuf.ptr; break;
-    case 6: src = h->hbuf.ptr; break;
-    case 7: src = h->yb.ptr; break;
-    case 8: src = (char*)h->kself + layer * self_layer; break;
-    case 9: src = (char*)h->vself + layer * self_layer; break;
-    case 12: src = h->mega_dbg; break;
-    default: return AD_ERR_ARG;
-  }
-  cudaStreamSynchronize(h->stream);
-  return cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? AD_OK : AD_ERR_CUDA;
-}
-#endif
 
 extern "C" int ad_debug_profile_verify(ad_handle* h, const int32_t* drafts, const int32_t* k, char* names, float* us,
                                        int32_t capacity, int32_t* n_launches) {

@@ -81,10 +81,6 @@ struct Params {
   int ring;                     // weight-ring depth (tiles)
   int b_bytes;                  // shared-memory area of a cluster stage's B operand; the reduction buffers follow it
   int red_bytes;                // one reduction buffer: (token capacity rounded up to 16) x 128 floats
-#ifdef AD_MEGA_DEBUG
-  int debug_stop;
-  float* dbg;      // [16 CTAs][32 stages][4]: sum |B operand|, sum |own partial|, jc, pb
-#endif
   unsigned long long* timeline; // optional: CTA 0 stamps the global timer when a stage's inputs are ready and when it has signalled
 };
 
@@ -105,11 +101,6 @@ struct Ctl {
   int red_idx[4][NT_MAX];
 };
 
-#ifdef AD_MEGA_DEBUG
-#define MEGA_STAMP(k) do { if (tid == 0 && g == 0 && s < 64) reinterpret_cast<long long*>(p.dbg + 4096)[s * 8 + (k)] = clock64(); } while (0)
-#else
-#define MEGA_STAMP(k) do { } while (0)
-#endif
 
 // ---- small PTX helpers -------------------------------------------------------------------------------------
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
@@ -457,11 +448,7 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
   const int G = gridDim.x, g = blockIdx.x, NC = G / CS, c = g / CS;
   const int R = p.ring;
   const int L = p.L;
-#ifdef AD_MEGA_DEBUG
-  const int n_stages = min(ST_PER_LAYER * L + 1, p.debug_stop);   // debugging builds can stop after a given stage
-#else
   const int n_stages = ST_PER_LAYER * L + 1;
-#endif
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t ring_base = smem_base;
   const uint32_t b_base = smem_base + (uint32_t)R * TILE_A;
@@ -617,7 +604,6 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
           if (!ok) break;
         }
         if (p.timeline && g == 0 && tid == 0) p.timeline[2 * s] = gs::now_ns();
-        MEGA_STAMP(0);
         // the x / statistics buffer holding this layer's input, and the other one
         const int in_buf = si.layer & 1, oth = in_buf ^ 1;
 
@@ -725,10 +711,8 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
               stage_b(p, ctl, bsrc, r * kpc, kpc, ntile, M, nullptr, b_base, nullptr, tid, nt == c ? stats_in : nullptr, M, bg, bb);
               __syncwarp();
               if (lane == 0) mbar_arrive_local(tc::smem_u32(&ctl->b_ready));
-              MEGA_STAMP(1);
               ok = worker_all(wait_bar(tc::smem_u32(&ctl->acc_full[a]), (jc >> 1) & 1, ctl, p.status));
               if (!ok) break;
-              MEGA_STAMP(2);
               asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
               // this CTA's partial [tokens x 128 features] -> reduction buffer pb
               float* red = red_ptr + (size_t)pb * (p.red_bytes / 4);
@@ -743,11 +727,9 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
               __syncwarp();
               if (lane == 0) mbar_arrive_local(tc::smem_u32(&ctl->acc_empty[a]));
               worker_sync();                                 // the whole partial is in shared memory
-              MEGA_STAMP(3);
               if (tid < CS) mbar_arrive_remote(tc::smem_u32(&ctl->red_full[pb]), (uint32_t)tid);
               ok = worker_all(wait_bar(tc::smem_u32(&ctl->red_full[pb]), (rc >> 1) & 1, ctl, p.status, true));
               if (!ok) break;
-              MEGA_STAMP(4);
               // sum the CS partials of this CTA's tokens in rank order; lane owns features 4 lane .. 4 lane + 3
               for (int tl_ = warp; tl_ < tpc; tl_ += 8) {
                 const int m = r * tpc + tl_;
@@ -791,7 +773,6 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
                   *reinterpret_cast<uint2*>(dst) = u;
                 }
               }
-              MEGA_STAMP(5);
               worker_sync();
               ++jc; ++rc;
             }
@@ -805,12 +786,8 @@ decoder_pass_kernel(const __grid_constant__ Params p) {
       __threadfence();
 #endif
       worker_sync();
-      MEGA_STAMP(6);
       if (tid == 0) {
         gs::arrive_release(p.sync_ctr + (size_t)s * SYNC_STRIDE, 1u);
-#ifdef AD_MEGA_DEBUG
-        if (g == 0 && s < 64) reinterpret_cast<long long*>(p.dbg + 4096)[s * 8 + 7] = clock64();
-#endif
         if (p.timeline && g == 0) p.timeline[2 * s + 1] = gs::now_ns();
       }
     }
