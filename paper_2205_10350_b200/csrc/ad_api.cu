@@ -131,6 +131,11 @@ struct ad_handle {
   int* down = nullptr;       // result block of finalize_generate_kernel (host view) ...
   int* down_dev = nullptr;   // ... and its device view
   bool defer_status = false; // ad_encode inside ad_generate: no synchronisation of its own
+  // Decode loop with small blocks: the accept kernel of iteration i also plans and embeds the block of iteration i + 1
+  // (loop_next.source >= 0), so an iteration starts at its first projection; pass_planned tells the pass being enqueued
+  // that its plan and embedding already exist.
+  NextBlock loop_next = {-1, 0, nullptr, 0, 0};
+  bool pass_planned = false;
   bool profiling = false;    // ad_debug_profile_verify: an event in front of every launch
   std::vector<std::pair<std::string, cudaEvent_t>> prof;
   // state
@@ -792,7 +797,7 @@ int decoder_pass(ad_handle* h, int pk, Model& m) {
   PassCfg& pc = h->pass[pk];
   const size_t self_layer = (size_t)h->dims.max_tgt * c.max_batch * c.d_model * h->esz;
   const size_t cross_layer = (size_t)c.max_src * c.max_batch * c.d_model * h->esz;
-  AD_TRY(embed(h, pc, m));
+  if (!(pk == PK_VERIFY && h->pass_planned)) AD_TRY(embed(h, pc, m));
   for (int l = 0; l < c.n_dec; ++l) {
     DecLayer& L = m.dec[l];
     void* kb = pk == PK_VERIFY ? (char*)h->kself + l * self_layer : h->ktmp;
@@ -874,10 +879,22 @@ int vocab_stage(ad_handle* h, Model& m, const ActBuf& X, int to_drafts, int auto
   }
   if (!partials_ready) AD_TRY(gemm(h, EPI_ARGMAX, m.emb, X, PK_VERIFY, pc.plan.M, pc.M_cap, p));
   note_launch(h, "argmax_accept");
-  AD_CUDA(h, launch_k(argmax_accept_kernel, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
-                      pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
-                      auto_commit ? h->cond_handle : 0ull, beta, h->tau, (const float*)h->draft_val, (const int*)h->draft_id,
-                      (const int*)h->part_cnt));
+  NextBlock nxt = {-1, 0, nullptr, 0, 0};
+  NextEmbed ne = {};
+  if (auto_commit && !to_drafts && h->loop_next.source >= 0) {
+    nxt = h->loop_next;
+    ne.emb = m.emb.ptr; ne.pe = h->pe; ne.d = h->cfg.d_model; ne.scale = sqrtf((float)h->cfg.d_model); ne.y = h->y; ne.yb = h->yb.ptr;
+  }
+  if (h->bf16)
+    AD_CUDA(h, launch_k(argmax_accept_kernel<bf16>, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
+                        pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
+                        auto_commit ? h->cond_handle : 0ull, beta, h->tau, (const float*)h->draft_val, (const int*)h->draft_id,
+                        (const int*)h->part_cnt, nxt, ne));
+  else
+    AD_CUDA(h, launch_k(argmax_accept_kernel<float>, dim3(h->dims.B), dim3(1024), 0, h->stream, h->st, pc.plan, h->dims, (const float*)h->part_val, (const int*)h->part_idx, h->n_vtiles,
+                        pc.M_cap, to_drafts, auto_commit, (unsigned int*)(h->st.loop_it + 1),
+                        auto_commit ? h->cond_handle : 0ull, beta, h->tau, (const float*)h->draft_val, (const int*)h->draft_id,
+                        (const int*)h->part_cnt, nxt, ne));
   h->last_vocab_which = to_drafts ? 1 : 0;
   return AD_OK;
 }
@@ -923,7 +940,29 @@ int commit_stage(ad_handle* h, const int* n_dev) {
 }
 
 // One iteration of the decode loop: draft -> verify -> commit, all on the device.
+// Whether the loop of these options lets the accept kernel plan and embed the next block: no drafter pass in between,
+// blocks small enough for one CTA to embed, kernel-chain form of the pass.
+bool g_fuse_plan = true;      // AD_NO_FUSED_PLAN=1: plan and embed as kernels of their own in every iteration
+bool loop_plans_ahead(const ad_handle* h, const ad_gen_opts& o) {
+  return g_fuse_plan && !(o.mode == AD_MODE_GAD && o.run_drafter) && h->pass[PK_VERIFY].M_cap <= 128 && !h->mega[PK_VERIFY].on;
+}
+
+// First block of a loop that plans ahead: planned and embedded by kernels of their own, before the loop.
+int plan_first_block(ad_handle* h, const ad_gen_opts& o, const int* ovr, int ovr_len) {
+  AD_TRY(prepare_verify(h, (o.mode == AD_MODE_GAD || ovr) ? SRC_OVERRIDE : SRC_POLICY, o.k, ovr, ovr_len));
+  return embed(h, h->pass[PK_VERIFY], h->ar);
+}
+
 int loop_iteration(ad_handle* h, const ad_gen_opts& o, const int* ovr, int ovr_len) {
+  if (loop_plans_ahead(h, o)) {
+    // this iteration's plan and embedding exist already (plan_first_block, or the previous iteration's accept kernel)
+    h->loop_next = NextBlock{(o.mode == AD_MODE_GAD || ovr) ? SRC_OVERRIDE : SRC_POLICY, o.k, ovr, h->cfg.max_tgt, ovr_len};
+    h->pass_planned = true;
+    const int rc = verify_stage(h, 1);
+    h->pass_planned = false;
+    h->loop_next.source = -1;
+    return rc;
+  }
   if (o.mode == AD_MODE_GAD) {
     if (o.run_drafter) {
       AD_TRY(draft_stage(h, o.k));
@@ -1001,6 +1040,7 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
   { const char* e = getenv("AD_NO_CONCURRENT_ENCODERS"); g_two_stream_encode = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_NO_ATTN_PROJ"); g_fuse_attn_proj = !(e && e[0] == '1'); }
   { const char* e = getenv("AD_MEGA"); g_use_mega = e && e[0] == '1'; }
+  { const char* e = getenv("AD_NO_FUSED_PLAN"); g_fuse_plan = !(e && e[0] == '1'); }
   if (major != 10) return fail(nullptr, AD_ERR_CUDA, "this library contains sm_100a code only; the current device is not compute capability 10.x");
 
   ad_handle* h = new ad_handle();
@@ -1396,6 +1436,7 @@ extern "C" int ad_generate(ad_handle* h, const int32_t* src, int32_t src_stride,
     }
   }
 
+  if (loop_plans_ahead(h, *opts)) AD_TRY(plan_first_block(h, *opts, ovr, ovr_len));
   if (device_loop) {
     // one launch runs every iteration; the data-independent bound on the iteration count travels in loop_it[3]
     h->host_flag[1] = max_iters + 1;

@@ -84,25 +84,29 @@ __device__ int warp_suffix_match(const int* out, int j, const int* src, int n, i
 // Chooses every row's block (size and drafted tokens) and lays the block tokens out as packed rows.
 // Decoder inputs of row b are (last accepted token, drafts[0..k-2]) at positions len .. len+k-1
 // (Eq. 6 / Eq. 7); a negative draft that would be fed is replaced by [PAD].
-// grid = 1, block = 256.
+// Executed by ALL threads of one CTA (any multiple of 32 threads); s_k / s_off: shared arrays of 256 / 257 ints.
+// The per-row state is read past L1: the caller may be the last CTA of the accept kernel, reading what the other
+// CTAs of that kernel have just committed.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap, const int* override_stream,
-                      int override_stride, int override_len) {
-  trace_mark(TR_PREPARE, 0);
-  pdl_launch();
-  pdl_wait();
-  trace_mark(TR_PREPARE, 1);
-  __shared__ int s_k[256];
-  __shared__ int s_off[257];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int B = dm.B;
+struct NextBlock {
+  int source;                  // DraftSource
+  int k_cap;
+  const int* override_stream;
+  int override_stride, override_len;
+};
+
+__device__ __forceinline__ void plan_verify_block(const DevState& st, const PassPlan& plan, const Dims& dm, const NextBlock& nb,
+                                                  int* s_k, int* s_off) {
+  const int tid = threadIdx.x, nthreads = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
+  const int B = dm.B, source = nb.source, k_cap = nb.k_cap;
+  const int* override_stream = nb.override_stream;
+  const int override_stride = nb.override_stride, override_len = nb.override_len;
 
   if (source == SRC_POLICY) {
-    for (int b = warp; b < B; b += 8) {
+    for (int b = warp; b < B; b += nwarps) {
       int k = 0;
-      const int len = st.len[b];
-      if (!st.fin[b] && len < st.maxlen[b]) {
+      const int len = __ldcg(st.len + b);
+      if (!__ldcg(st.fin + b) && len < st.maxlen[b]) {
         const int n = st.srclen[b];
         const int* src = st.src + (size_t)b * dm.max_src;
         const int i = warp_suffix_match(st.out_ids + (size_t)b * dm.max_tgt, len, src, n, dm.bos, lane);
@@ -120,16 +124,16 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
       if (lane == 0) s_k[b] = k;
     }
   } else {
-    for (int b = tid; b < B; b += 256) {
+    for (int b = tid; b < B; b += nthreads) {
       int k;
-      const int len = st.len[b];
+      const int len = __ldcg(st.len + b);
       if (source == SRC_USER) {
         k = st.user_k[b];
         if (k < 0 || k > dm.kmax || len + k > dm.max_tgt) { latch_error(st.status, AD_ERR_ARG); k = 0; }
       } else if (source == SRC_KEEP) {
         k = plan.seg_len[b];
       } else {
-        k = (st.fin[b] || len >= st.maxlen[b]) ? 0 : min(k_cap, st.maxlen[b] - len);
+        k = (__ldcg(st.fin + b) || len >= st.maxlen[b]) ? 0 : min(k_cap, st.maxlen[b] - len);
       }
       s_k[b] = k;
     }
@@ -144,8 +148,8 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
   }
   if (tid < 128) st.sync_ctr[tid * 32] = 0u;
   __syncthreads();
-  for (int b = warp; b < B; b += 8) {
-    const int k = s_k[b], off = s_off[b], len = st.len[b];
+  for (int b = warp; b < B; b += nwarps) {
+    const int k = s_k[b], off = s_off[b], len = __ldcg(st.len + b);
     int* dr = st.drafts + (size_t)b * dm.kmax;
     if (lane == 0) {
       plan.seg_off[b] = off;
@@ -163,7 +167,7 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
     __syncwarp();
     for (int i = lane; i < k; i += 32) {
       const int m = off + i;
-      int tok = (i == 0) ? st.last[b] : dr[i - 1];
+      int tok = (i == 0) ? __ldcg(st.last + b) : dr[i - 1];
       if (tok < 0 || tok >= dm.vocab) tok = dm.pad;
       plan.tok_row[m] = b;
       plan.tok_pos[m] = len + i;
@@ -172,6 +176,22 @@ prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap
       plan.att_n[m] = len + i + 1;
     }
   }
+}
+
+// grid = 1, block = 256.
+__global__ void __launch_bounds__(256)
+prepare_verify_kernel(DevState st, PassPlan plan, Dims dm, int source, int k_cap, const int* override_stream,
+                      int override_stride, int override_len) {
+  trace_mark(TR_PREPARE, 0);
+  pdl_launch();
+  pdl_wait();
+  trace_mark(TR_PREPARE, 1);
+  __shared__ int s_k[256];
+  __shared__ int s_off[257];
+  NextBlock nb;
+  nb.source = source; nb.k_cap = k_cap; nb.override_stream = override_stream;
+  nb.override_stride = override_stride; nb.override_len = override_len;
+  plan_verify_block(st, plan, dm, nb, s_k, s_off);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -579,14 +599,30 @@ draft_score_kernel(DevState st, PassPlan blk, Dims dm, const WT* __restrict__ em
 // auto_commit != 0: the row's n_accepted is committed right away (decode loop); the last CTA to finish
 //   updates the loop counter and the all-finished word (done_ctr: rows done in the low half, active rows in
 //   the high half; left at zero).
+// next.source >= 0 (decode loop, small blocks): the LAST CTA to finish also chooses the next iteration's blocks
+//   (plan_verify_block) and embeds their tokens (y = emb[token] * sqrt(d) + PE[pos]), so that the next iteration starts
+//   at its first projection: two launches fewer per iteration.
 // grid = B, block = 1024.
 // ---------------------------------------------------------------------------------------------
+struct NextEmbed {
+  const void* emb;       // embedding matrix in the weight type
+  const float* pe;
+  int d;
+  float scale;
+  float* y;
+  void* yb;              // GEMM-operand copy in the activation type
+};
+
+template <typename WT>
 __global__ void __launch_bounds__(1024)
 argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict__ part_val,
                      const int* __restrict__ part_idx, int n_tiles, int M_cap, int to_drafts, int auto_commit,
                      unsigned int* done_ctr, unsigned long long cond, int beta, float tau,
                      const float* __restrict__ draft_val, const int* __restrict__ draft_id,
-                     const int* __restrict__ part_cnt) {
+                     const int* __restrict__ part_cnt, NextBlock next, NextEmbed ne) {
+  __shared__ int s_k[256];
+  __shared__ int s_off[257];
+  __shared__ int s_last;
   trace_mark(TR_ACCEPT, 0);
   pdl_launch();
   pdl_wait();
@@ -627,6 +663,7 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
     }
   }
   if (to_drafts) return;
+  if (tid == 0) s_last = 0;
   __syncthreads();
   if (warp == 0) {
     int n = 0;
@@ -659,7 +696,30 @@ argmax_accept_kernel(DevState st, PassPlan blk, Dims dm, const float* __restrict
           __threadfence();
           finish_iteration(st, dm, ((t >> 16) + (n > 0 ? 1u : 0u)) != 0, cond);
           *done_ctr = 0;
+          s_last = 1;
         }
+      }
+    }
+  }
+  if (auto_commit && next.source >= 0) {
+    __syncthreads();
+    if (s_last) {                  // block-uniform: this CTA saw every row committed
+      __threadfence();
+      plan_verify_block(st, blk, dm, next, s_k, s_off);
+      __syncthreads();
+      // embedding of the next block's tokens (written by this CTA just above)
+      const int M = s_off[dm.B], d = ne.d, groups = d >> 2;
+      const WT* emb = reinterpret_cast<const WT*>(ne.emb);
+      WT* yb = reinterpret_cast<WT*>(ne.yb);
+      for (int idx = tid; idx < M * groups; idx += blockDim.x) {
+        const int m = idx / groups, c = (idx - m * groups) * 4;
+        const WT* er = emb + (size_t)blk.tok_id[m] * d + c;
+        const float4 pp = *reinterpret_cast<const float4*>(ne.pe + (size_t)blk.tok_pos[m] * d + c);
+        float4 v;
+        v.x = to_f32(er[0]) * ne.scale + pp.x; v.y = to_f32(er[1]) * ne.scale + pp.y;
+        v.z = to_f32(er[2]) * ne.scale + pp.z; v.w = to_f32(er[3]) * ne.scale + pp.w;
+        *reinterpret_cast<float4*>(ne.y + (size_t)m * d + c) = v;
+        store4(yb + (size_t)m * d + c, v);
       }
     }
   }
