@@ -49,3 +49,19 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                         "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_algorithmic_bytes_of_a_verification_step():
+    """The byte counts behind the bench line's roofline: per-step weight bytes Ld(6d^2 + 2dF)s + Vds for the three model
+    sizes (cross-attention K/V projections excluded: they run once per sentence), and the key/value terms of a step."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2205_10350_b200 import synth
+    assert bench.weight_bytes(synth.BASE) == 38_404_096 * 2 == 76_808_192
+    assert bench.weight_bytes(synth.BIG) == 120_848_384 * 2
+    assert bench.weight_bytes(synth.TINY) == 586_752 * 4
+    # one base-model step: 32 source tokens, a 16-token block on a 16-token prefix: 12 288 bytes per key/value token
+    per_tok = 2 * 6 * 512 * 2
+    assert per_tok == 12_288
+    assert bench.step_bytes(synth.BASE, 32, 32, 16) == 76_808_192 + per_tok * (32 + 32 + 16)
+    assert bench.step_bytes(synth.BASE, 0, 0, 0, n_steps=3) == 3 * 76_808_192
