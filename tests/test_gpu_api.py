@@ -255,3 +255,20 @@ def test_grid_barrier_passes_data_and_its_bounded_wait_runs_out():
     assert int(status.item()) == binding.AD_ERR_TIMEOUT and result.cpu().numpy()[1] == 0
     x = torch.ones((4, 64), device="cuda:0").bfloat16()
     assert float(binding.linear(x, x)[0, 0]) == 64.0
+
+
+def test_per_kernel_profile_of_a_block_changes_nothing(setup):
+    """ad_debug_profile_verify: the block is verified as usual (same ids and accepted length as ad_verify_block), and every
+    launch comes back with a name and a positive device time."""
+    dec, om = setup
+    src = np.array([[5, 6, 7, 8, 9, 10, 11, 12, 13, 14]], np.int32)
+    dec.encode(src, [10])
+    drafts = np.array([[20, 21, 22, 23, 24, 25]], np.int32)
+    ids, n = dec.verify_block(drafts, [6])
+    prof = dec.profile_verify(drafts, [6])
+    ids2, n2 = dec.verify_block(drafts, [6])
+    assert np.array_equal(ids, ids2) and n[0] == n2[0]
+    names = [p[0] for p in prof]
+    assert len(prof) >= 10 and all(us > 0 for _, us in prof)
+    assert names[0] == "prepare_verify" and "embed" in names and any(x.startswith("gemm_") for x in names)
+    assert names[-1] in ("argmax_accept", "ad_verify_block")
