@@ -141,6 +141,13 @@ def main():
             dec.sync()
             out.update(model=args.model, batch=B, k=args.k, prefix=args.prefix, src=args.src,
                        us_mean=statistics.mean(ts), us_min=min(ts), launch="direct (no graph)")
+            import os
+            if os.environ.get("AD_MEGA") == "1" and os.environ.get("AD_MEGA_TIMELINE") == "1":
+                # persistent decoder pass: per stage (inputs visible, signalled) stamps of CTA 0, last step
+                tl = dec.debug_stage_timeline().astype(np.int64)
+                t0 = int(tl[0, 0])
+                out["stage_ready_us"] = [round(1e-3 * (int(a) - t0), 2) for a, _ in tl]
+                out["stage_busy_us"] = [round(1e-3 * (int(b) - int(a)), 2) for a, b in tl]
         else:
             tot_it, tot_ms, tot_tok, launches = 0, 0.0, 0, 0
             for s in range(args.sentences):
