@@ -77,6 +77,30 @@ def reduce_max_sum(dist, dev, seconds_or_ms, count):
     return float(t.item()), int(n.item())
 
 
+# DRAM counters of one verification step (dram__bytes_read.sum + dram__bytes_write.sum summed over the step's
+# kernels, ncu, caches flushed before every kernel) with the digest of the kernel sources they were taken on:
+# the figures are reported only while the sources still have that digest.
+NCU_COUNTERS = dict(sources_sha256="93fc91734be7bdb3f029bce8116b3b8a11b443a5d49ae86d7bfad021bcfc291c",
+                    step_block40_bytes=102940160, projection_bytes=32862000,
+                    summary="profiles/verify_step_base_b1_k40_dram_traffic.txt")
+
+
+def kernel_sources_digest():
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2205_10350_b200", "csrc", "*"))):
+        h.update(os.path.basename(path).encode())
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_counter(key):
+    """The stored counter, or None once a kernel source has changed since it was taken."""
+    return NCU_COUNTERS[key] if kernel_sources_digest() == NCU_COUNTERS["sources_sha256"] else None
+
+
 def weight_bytes(shape):
     """Algorithmic weight bytes of one verification step: decoder layers (cross-attention K/V projections excluded:
     they run once per sentence in the encoder pass) + the output projection."""
@@ -454,11 +478,13 @@ def run_ours(args, rank, world, local_rank):
     wv = weight_bytes(synth.BASE)
     roofline = dict(bound="hbm", kernel="verification step: the 56-kernel chain of one loop iteration (6 decoder layers of 9 kernels, "
                     "projection + arg-max, accept + commit + plan and embedding of the next block), graph-replayed", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
-                    frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"], algorithmic_bytes=alg,
+                    frac=ach / pk["hbm_gbs"], traffic=ncu_counter("step_block40_bytes"), peak_source=pk["source"], algorithmic_bytes=alg,
                     weight_bytes=wv, us_per_step_in_loop=loop_us, hbm_floor_us=alg / (pk["hbm_gbs"] * 1e9) * 1e6,
                     note="time = device time of the decode loops / loop iterations (weights L2-warm between the iterations of a "
-                         "sentence, L2 flushed between timed steps); traffic is null because the step is a chain of kernels, "
-                         "none of which dominates: see `kernels` and profiles/ for the per-kernel DRAM counters")
+                         "sentence, L2 flushed between timed steps); traffic = DRAM bytes summed over the kernels of one 40-token "
+                         "step on an empty prefix, every kernel measured with cold caches (" + NCU_COUNTERS["summary"] + "): the "
+                         "weights (76.8 MB) once, plus the activations handed from kernel to kernel, which in the running chain "
+                         "stay in L2; null once a kernel source has changed since the capture")
     out_line = dict(value=value, t_ms=t_ms, tokens=tokens, e2e=dict(value=e2e_tok / e2e_t, unit=UNIT, h2d_bytes_per_step=h2d,
                                                                    d2h_bytes_per_step=d2h),
                     clocks=clocks, agg=agg, iters=iters, roofline=roofline, it_per_sent=it_per_sent)
@@ -518,8 +544,9 @@ def bench_extras(args, binding, dec, w, dev, pk, flush, t_src, t_len, t_max, t_o
     extras["projection_kernel"] = dict(kernel="gemm_tc_kernel<EPI_ARGMAX>, vocabulary 32000 x 512, 40 tokens", algorithmic_bytes=vb,
                                        us_cold=t_cold, us_l2_warm=t_warm, gbs_cold=vb / (t_cold * 1e-6) / 1e9,
                                        frac_of_hbm_peak_cold=vb / (t_cold * 1e-6) / 1e9 / pk["hbm_gbs"],
-                                       traffic_ncu=32855040, traffic_note="dram__bytes_read.sum + dram__bytes_write.sum of one launch "
-                                       "(profiles/vocab_argmax_gemm_base_M40_ncu_full.txt; this kernel is unchanged since that capture)")
+                                       traffic_ncu=ncu_counter("projection_bytes"),
+                                       traffic_note="dram__bytes_read.sum + dram__bytes_write.sum of one launch (" +
+                                       NCU_COUNTERS["summary"] + "); null once a kernel source has changed since the capture")
 
     # fixed-shape verification steps, weight-streaming regime (direct launches): L2-warm and L2-flushed
     pts = []

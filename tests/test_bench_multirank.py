@@ -65,3 +65,17 @@ def test_algorithmic_bytes_of_a_verification_step():
     assert per_tok == 12_288
     assert bench.step_bytes(synth.BASE, 32, 32, 16) == 76_808_192 + per_tok * (32 + 32 + 16)
     assert bench.step_bytes(synth.BASE, 0, 0, 0, n_steps=3) == 3 * 76_808_192
+
+
+def test_stored_profiler_counters_expire_with_the_kernel_sources(monkeypatch):
+    """The DRAM counters the bench line repeats were taken on one state of the kernel sources: they are reported while
+    the sources hash to the stored digest and become null otherwise."""
+    sys.path.insert(0, ROOT)
+    import bench
+    digest = bench.kernel_sources_digest()
+    assert len(digest) == 64 and digest == bench.kernel_sources_digest()
+    monkeypatch.setitem(bench.NCU_COUNTERS, "sources_sha256", digest)
+    assert bench.ncu_counter("step_block40_bytes") == bench.NCU_COUNTERS["step_block40_bytes"] > bench.weight_bytes(
+        __import__("paper_2205_10350_b200.synth", fromlist=["BASE"]).BASE)
+    monkeypatch.setitem(bench.NCU_COUNTERS, "sources_sha256", "0" * 64)
+    assert bench.ncu_counter("step_block40_bytes") is None and bench.ncu_counter("projection_bytes") is None
