@@ -263,7 +263,8 @@ int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32_t absent_c
 /* Output projection fused with the row arg-max (Eq. 3 / Eq. 7 "top-1"): for each of M rows of x [M, d]
  * (dtype as given) against emb [vocab, d], argmax[m] = lowest id with the largest score; the scores are
  * never written.  scratch: device memory for per-tile partial maxima, ad_vocab_argmax_scratch_bytes().
- * status: optional device int that latches AD_ERR_TIMEOUT.  BF16 needs d % 64 == 0 and M <= 256.
+ * status: optional device int that latches AD_ERR_TIMEOUT.  BF16 needs d % 64 == 0 and M <= 65536 (more than
+ * 256 rows run as 256-token tiles).
  * argmax == NULL runs the projection kernel alone and leaves its per-tile (maximum, id) partials in scratch
  * (values [M, tiles] FP32 first, ids [M, tiles] int32 from the next 256-byte boundary, tiles = ceil(vocab / 128)):
  * the launch a micro-benchmark times when it wants the projection without the final reduction. */
@@ -297,7 +298,7 @@ int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dtype, int32_
                            int32_t* argmax, int32_t* status, void* stream);
 
 /* y [M, N] (FP32) = x [M, K] W^T + bias, W [N, K] in `dtype` (Section 2 projections).  bias may be NULL.
- * BF16 needs K % 64 == 0 and M <= 256. */
+ * BF16 needs K % 64 == 0 and M <= 65536. */
 int ad_linear(const void* x, const void* W, const float* bias, int32_t dtype, int32_t M, int32_t K,
               int32_t N, float* y, int32_t* status, void* stream);
 

@@ -1662,6 +1662,10 @@ extern "C" int ad_debug_grid_barrier_probe(int32_t n_ctas, int32_t rounds, int32
 
 // ---- single-kernel entry points -----------------------------------------------------------------
 
+namespace {
+constexpr int kMaxOpTokens = 65536;   // operator-level entries: token rows per call (256-token tiles along grid.y)
+}
+
 extern "C" size_t ad_vocab_argmax_scratch_bytes(int32_t vocab, int32_t M) {
   const size_t tiles = (size_t)(vocab + 127) / 128;
   return align_up(tiles * (size_t)M * sizeof(float), 256) + align_up(tiles * (size_t)M * sizeof(int), 256);
@@ -1700,7 +1704,7 @@ extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, in
   p.K = d; p.N = vocab; p.M_ptr = nullptr; p.M_host = M; p.M_cap = M; p.part_val = pv; p.part_idx = pi; p.status = status;
   cudaError_t e;
   if (dtype == AD_DTYPE_BF16) {
-    if (d % 64 || M > 256) return AD_ERR_ARG;
+    if (d % 64 || M > kMaxOpTokens) return AD_ERR_ARG;
     CUtensorMap mw, mx;
     p.ntile = clampi(pow2ceil(M), 16, 256);
     if (!make_map(&mw, emb, vocab, d, tc::BLOCK_N_FEAT) || !make_map(&mx, x, M, d, p.ntile)) return AD_ERR_CUDA;
@@ -1725,7 +1729,7 @@ extern "C" int ad_linear(const void* x, const void* W, const float* bias, int32_
   p.K = K; p.N = N; p.M_ptr = nullptr; p.M_host = M; p.M_cap = M; p.bias = bias; p.out_f32 = y; p.status = status;
   cudaError_t e;
   if (dtype == AD_DTYPE_BF16) {
-    if (K % 64 || M > 256) return AD_ERR_ARG;
+    if (K % 64 || M > kMaxOpTokens) return AD_ERR_ARG;
     CUtensorMap mw, mx;
     p.ntile = clampi(pow2ceil(M), 16, 256);
     if (!make_map(&mw, W, N, K, tc::BLOCK_N_FEAT) || !make_map(&mx, x, M, K, p.ntile)) return AD_ERR_CUDA;
@@ -1768,7 +1772,7 @@ extern "C" int ad_vocab_argmax_static(const void* x, const void* emb, int32_t dt
   }
   const int rc = ad_vocab_argmax(x, emb, dtype, M, d, vocab, argmax, g_static_scratch_addr[dev], AD_STATIC_SCRATCH_BYTES, status, stream);
   if (rc != AD_OK)
-    return fail(nullptr, rc, rc == AD_ERR_ARG ? "ad_vocab_argmax_static: unsupported shape or dtype (BF16 needs d % 64 == 0 and M <= 256)"
+    return fail(nullptr, rc, rc == AD_ERR_ARG ? "ad_vocab_argmax_static: unsupported shape or dtype (BF16 needs d % 64 == 0 and M <= 65536)"
                                               : "ad_vocab_argmax_static: encoding a TMA descriptor or launching a kernel failed");
   return AD_OK;
 }

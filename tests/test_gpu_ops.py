@@ -80,3 +80,30 @@ def test_argmax_ties_go_to_the_lowest_id():
     assert (got == 131).all()
     got = binding.vocab_argmax(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(E, device=DEV).bfloat16()).cpu().numpy()
     assert (got == 131).all()
+
+
+def test_tensor_regime_sizes_on_sampled_rows():
+    """2048 packed tokens (batch 32 x block 64 of the base model), the size the batched benchmark point runs at:
+    256-token tiles, two CTAs per SM, several waves.  The checker computes a sample of token rows (first and last rows
+    of tiles, the last row of the pass) of the QKV-sized and FFN-sized projections and of the fused projection +
+    arg-max."""
+    M, d, V = 2048, 512, 32000
+    rows = np.array([0, 1, 127, 128, 255, 256, 1023, 1024, 1500, 1791, 1792, 2046, 2047])
+    for (K, N) in ((d, 3 * d), (d, 4 * d), (4 * d, d)):
+        x, W, b = _data(M, K, N, True, seed=K + N)
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        y = binding.linear(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(W, device=DEV).bfloat16(),
+                           torch.tensor(b, device=DEV), st).cpu().numpy()
+        ref = OPS.linear(x[rows].copy(), W.T.copy(), b)
+        assert np.abs(y[rows] - ref).max() < 2e-4 * max(1.0, np.abs(ref).max())
+        assert int(st.item()) == 0 and np.isfinite(y).all()
+    r = np.random.default_rng(11)
+    x = synth.round_to_bf16(r.standard_normal((M, d)).astype(np.float32))
+    E = synth.round_to_bf16((r.standard_normal((V, d)) * 0.02).astype(np.float32))
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    got = binding.vocab_argmax(torch.tensor(x, device=DEV).bfloat16(), torch.tensor(E, device=DEV).bfloat16(), st).cpu().numpy()
+    assert got.shape == (M,) and int(st.item()) == 0 and (got >= 0).all() and (got < V).all()
+    lg = OPS.linear(x[rows].copy(), E.T.copy(), None)
+    for j, m in enumerate(rows):
+        i1, v1, i2, v2 = OPS.top2(lg[j])
+        assert got[m] == i1 if v1 - v2 > 1e-4 else got[m] in (i1, i2)
