@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libad_b200.so")
 SOURCES = ["ad_api.cu"]
-HEADERS = ["ad_common.cuh", "gemm_tc.cuh", "gemm_simt.cuh", "attention.cuh", "attention_mma.cuh", "steps.cuh", "grid_sync.cuh", "mega.cuh"]
+HEADERS = ["ad_common.cuh", "gemm_tc.cuh", "gemm_tc_persistent.cuh", "gemm_simt.cuh", "attention.cuh", "attention_mma.cuh", "steps.cuh", "grid_sync.cuh", "mega.cuh"]
 
 
 def _stale() -> bool:

@@ -15,6 +15,7 @@
 #include "attention_mma.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc_persistent.cuh"
 #include "grid_sync.cuh"
 #include "mega.cuh"
 #include "steps.cuh"
@@ -478,6 +479,33 @@ cudaError_t launch_tc(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap&
   return launch_k(tc::gemm_tc_kernel<EPI>, grid, dim3(tc::THREADS), smem, st, mw, mx, p, stages);
 }
 
+// Projection + arg-max over many tokens: the persistent token-stationary kernel (one CTA per SM, 128-token tiles
+// resident in shared memory, read-out of one tile under the K loop of the next) once there are at least `min_pairs_per_sm`
+// (128 token x 256 vocabulary row) pairs per SM; AD_NO_PERSISTENT_VOCAB=1 keeps the one-tile-per-CTA kernel.
+bool vocab_goes_persistent(int K, int N, int M_cap, const float* bias) {
+  static const bool enabled = [] { const char* e = getenv("AD_NO_PERSISTENT_VOCAB"); return !(e && e[0] == '1'); }();
+  if (!enabled || bias || K % tc::BLOCK_K || K / tc::BLOCK_K > tc::P_MAX_KB) return false;
+  const long pairs = (long)((N + tc::P_VOC - 1) / tc::P_VOC) * ((M_cap + tc::P_TOK - 1) / tc::P_TOK);
+  return pairs >= (long)num_sms();
+}
+// mx128: the token operand's map with a 128-row box.
+cudaError_t launch_vocab_persistent(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx128, const GemmParams& p, int M_cap) {
+  static bool attr_set[kMaxDevices] = {};
+  const int dev = current_device();
+  constexpr int kSmemLimit = 227 * 1024 - 512;   // the kernel's static shared memory is a few hundred bytes
+  if (!attr_set[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(tc::vocab_argmax_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    if (e != cudaSuccess) return e;
+    attr_set[dev] = true;
+  }
+  const int kb = p.K / tc::BLOCK_K;
+  const int stages = clampi((kSmemLimit - 1024 - kb * tc::P_A_KB_BYTES) / tc::P_B_STAGE_BYTES, 1, tc::P_MAX_STAGES);
+  const long pairs = (long)((p.N + tc::P_VOC - 1) / tc::P_VOC) * ((M_cap + tc::P_TOK - 1) / tc::P_TOK);
+  const int grid = (int)std::min<long>(pairs, num_sms());
+  return launch_k(tc::vocab_argmax_persistent_kernel, dim3(grid), dim3(tc::P_THREADS), tc::vocab_persistent_smem(kb, stages), st, mw, mx128, p,
+                  stages);
+}
+
 template <int EPI>
 cudaError_t launch_simt(cudaStream_t st, const void* w, const void* x, const GemmParams& p, int M_cap) {
   dim3 grid((p.N + 127) / 128, (M_cap + simt::TOK - 1) / simt::TOK);
@@ -501,7 +529,12 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
       case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, mx, p, M_cap); break;
       case EPI_ACT: e = launch_tc<EPI_ACT>(h->stream, W.map, mx, p, M_cap); break;
       case EPI_SCATTER: e = launch_tc<EPI_SCATTER>(h->stream, W.map, mx, p, M_cap); break;
-      default: e = launch_tc<EPI_ARGMAX>(h->stream, W.map, mx, p, M_cap); break;
+      default:
+        // (a pass with a 256-token tile also has the 128-row map of its token operand)
+        e = (h->pass[pk].ntile == 256 && vocab_goes_persistent(W.K, W.N, M_cap, p.bias))
+                ? launch_vocab_persistent(h->stream, W.map, X.map_half[pk], p, M_cap)
+                : launch_tc<EPI_ARGMAX>(h->stream, W.map, mx, p, M_cap);
+        break;
     }
   } else {
     p.ntile = simt::TOK;
@@ -1708,7 +1741,13 @@ extern "C" int ad_vocab_argmax(const void* x, const void* emb, int32_t dtype, in
     CUtensorMap mw, mx;
     p.ntile = clampi(pow2ceil(M), 16, 256);
     if (!make_map(&mw, emb, vocab, d, tc::BLOCK_N_FEAT) || !make_map(&mx, x, M, d, p.ntile)) return AD_ERR_CUDA;
-    e = launch_tc<EPI_ARGMAX>(st, mw, mx, p, M);
+    if (vocab_goes_persistent(d, vocab, M, nullptr)) {
+      CUtensorMap mx128;
+      if (!make_map(&mx128, x, M, d, tc::P_TOK)) return AD_ERR_CUDA;
+      e = launch_vocab_persistent(st, mw, mx128, p, M);
+    } else {
+      e = launch_tc<EPI_ARGMAX>(st, mw, mx, p, M);
+    }
   } else if (dtype == AD_DTYPE_FP32) {
     p.ntile = simt::TOK;
     e = launch_simt<EPI_ARGMAX>(st, emb, x, p, M);

@@ -105,10 +105,21 @@ __device__ __forceinline__ void trace_mark(int id, int phase) {
     if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)(id * 8 + phase) << 56);
   }
 }
+// The same from whichever thread of CTA 0 calls it (role threads of warp-specialised kernels).
+__device__ __forceinline__ void trace_mark_role(int id, int phase) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const unsigned int i = atomicAdd(&g_trace_n, 1u);
+    if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)(id * 8 + phase) << 56);
+  }
+}
 #else
 __device__ __forceinline__ void trace_mark(int, int) {}
+__device__ __forceinline__ void trace_mark_role(int, int) {}
 #endif
-enum TraceId { TR_GEMM = 0, TR_ATTN = 8, TR_LN = 9, TR_EMBED = 10, TR_PREPARE = 11, TR_ACCEPT = 12, TR_COMMIT = 13 };
+enum TraceId { TR_GEMM = 0, TR_ATTN = 8, TR_LN = 9, TR_EMBED = 10, TR_PREPARE = 11, TR_ACCEPT = 12, TR_COMMIT = 13,
+               TR_PV_ISSUE = 20, TR_PV_EPI = 21, TR_PV_LOAD = 22 };
 
 __device__ __forceinline__ void latch_error(int* status, int code) {
   if (status) atomicCAS(status, 0, code);

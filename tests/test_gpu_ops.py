@@ -49,7 +49,10 @@ def test_bf16_tensor_core_linear(M, K, N):
 
 
 @pytest.mark.parametrize("bf16,M,d,V", [(False, 9, 128, 1000), (True, 40, 512, 32000), (True, 64, 1024, 4100),
-                                        (True, 1, 512, 32000), (True, 130, 256, 2048)])
+                                        (True, 1, 512, 32000), (True, 130, 256, 2048),
+                                        # many tokens (token-stationary kernel): ragged last vocabulary tile, then a
+                                        # vocabulary whose last 256-row pair has an empty second half; ragged token tile
+                                        (True, 1000, 256, 5000), (True, 1000, 256, 4900), (True, 300, 512, 32000)])
 def test_projection_with_fused_argmax(bf16, M, d, V):
     r = np.random.default_rng(4)
     x = r.standard_normal((M, d)).astype(np.float32)
