@@ -579,7 +579,33 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   p.scale = 1.0f / sqrtf((float)dh);
   // Tensor-core kernel when there are thousands of queries or rows may hold hundreds of keys (max_keys: the
   // capacity, known on the host); the FFMA kernel spreads few queries and few keys over more CTAs.
-  if (h->bf16 && dh == 64 && (many || max_keys >= 256)) {
+  if (h->bf16 && dh == 64 && max_keys >= 256) {
+    // rows may hold hundreds of keys: the keys of a row are spread over the warps of a CTA (whole 64-key tiles per warp),
+    // 1, 2 or 4 query tiles of 16 per CTA depending on how many queries a row can have
+    const int qt = pc.seg_max <= 16 ? 1 : (pc.seg_max <= 32 ? 2 : 4);
+    const int nw = qt == 4 ? 4 : 8;
+    p.qchunks = (pc.seg_max + 16 * qt - 1) / (16 * qt);
+    note_launch(h, "attention_mma_wide");
+    const dim3 mgrid(h->dims.B * p.qchunks, c.n_heads);
+    const size_t smem = (size_t)nw * AM_TILE_BYTES + AM_Q_BYTES;
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device();
+    cudaError_t em = cudaSuccess;
+    if (!attr_set[dev]) {
+      em = cudaFuncSetAttribute(attention_mma_wide_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * AM_TILE_BYTES + AM_Q_BYTES);
+      if (em == cudaSuccess) em = cudaFuncSetAttribute(attention_mma_wide_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * AM_TILE_BYTES + AM_Q_BYTES);
+      if (em == cudaSuccess) em = cudaFuncSetAttribute(attention_mma_wide_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * AM_TILE_BYTES + AM_Q_BYTES);
+      if (em != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention attribute: ") + cudaGetErrorString(em));
+      attr_set[dev] = true;
+    }
+    if (qt == 1) em = launch_k(attention_mma_wide_kernel<1, 8>, mgrid, dim3(256), smem, h->stream, p);
+    else if (qt == 2) em = launch_k(attention_mma_wide_kernel<2, 8>, mgrid, dim3(512), smem, h->stream, p);
+    else em = launch_k(attention_mma_wide_kernel<4, 4>, mgrid, dim3(512), smem, h->stream, p);
+    if (em != cudaSuccess) return fail(h, AD_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(em));
+    return AD_OK;
+  }
+  // Tensor-core kernel when there are thousands of queries; the FFMA kernel spreads few queries and few keys over more CTAs.
+  if (h->bf16 && dh == 64 && many) {
     // rows with few queries: warps share a 16-query tile and split the keys (2 or 4 key groups)
     const int ng = pc.seg_max <= 16 ? 4 : (pc.seg_max <= 32 ? 2 : 1);
     const int qcta = AM_Q / ng;
