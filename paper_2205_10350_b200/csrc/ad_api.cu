@@ -76,7 +76,11 @@ struct PassCfg {
     const int tiles = ((N + 127) / 128) * ((M_cap + tile - 1) / tile);
     const int kb = K / 64;
     int s = 1;
-    while (s * 2 <= max_split && tiles * s * 2 <= 160 && kb % (s * 2) == 0) s *= 2;
+    // Few tokens (one or two token tiles): at most ~3/4 of the SMs.  Measured, a 128-CTA split-K grid of these
+    // one-CTA-per-SM kernels ran 16 of its CTAs as a second wave behind the predecessor it overlaps (9.5 us instead of
+    // 5.3 us).  With many tokens the grid has several waves anyway and the split keeps the K loops short.
+    const int cap = M_cap <= 256 ? 112 : 160;
+    while (s * 2 <= max_split && tiles * s * 2 <= cap && kb % (s * 2) == 0) s *= 2;
     return s;
   }
 };
@@ -549,17 +553,17 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   return AD_OK;
 }
 
-template <typename T, int D, int Q, bool FUSE = false>
+template <typename T, int D, int Q, bool FUSE = false, int MINB = 1>
 cudaError_t launch_attention(dim3 grid, dim3 block, cudaStream_t st, const AttnParams& p) {
   constexpr size_t smem = att_smem_bytes<D, Q>();
   static bool attr_set[kMaxDevices] = {};
   const int dev = current_device();
   if (!attr_set[dev] && smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<T, D, Q, FUSE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   attr_set[dev] = true;
-  return launch_k(attention_kernel<T, D, Q, FUSE>, grid, block, smem, st, p);
+  return launch_k(attention_kernel<T, D, Q, FUSE, MINB>, grid, block, smem, st, p);
 }
 
 int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, const void* v, void* out,
@@ -632,7 +636,9 @@ int attention(ad_handle* h, const PassCfg& pc, const void* q, const void* k, con
   note_launch(h, fuse ? "attention+out_proj" : "attention");
   if (fuse) {
     p.wo = (const bf16*)wo->ptr; p.o_part = h->pre2; p.o_stride = (size_t)pc.M_cap * c.d_model;
-    e = launch_attention<bf16, 64, 1, true>(grid, block, h->stream, p);
+    // more CTAs than SMs: the two-CTAs-per-SM build, so that the grid is still one wave
+    e = (long)grid.x * grid.y > num_sms() ? launch_attention<bf16, 64, 1, true, 2>(grid, block, h->stream, p)
+                                           : launch_attention<bf16, 64, 1, true, 1>(grid, block, h->stream, p);
   } else if (h->bf16) {
     if (dh == 64) e = many ? AD_ATT(bf16, 64, 8) : AD_ATT(bf16, 64, 1);
     else e = many ? AD_ATT(bf16, 32, 8) : AD_ATT(bf16, 32, 1);

@@ -97,6 +97,16 @@ __device__ unsigned long long g_trace_buf[1 << 15];
 __device__ unsigned int g_trace_n;
 __device__ __forceinline__ void trace_mark(int id, int phase) {
   const bool first = blockIdx.x == 0, last = blockIdx.x == gridDim.x - 1 && gridDim.x > 1;
+#ifdef AD_TRACE_ALL_EXITS
+  // every CTA stamps its exit (under id + 16 unless it is CTA (0,0,0)): shows the tail of a grid
+  if (phase == 2 && threadIdx.x == 0 && !(first && blockIdx.y == 0 && blockIdx.z == 0)) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const unsigned int i = atomicAdd(&g_trace_n, 1u);
+    if (i < (1u << 15)) g_trace_buf[i] = (t & 0x00FFFFFFFFFFFFFFull) | ((unsigned long long)((id + 16) * 8 + phase) << 56);
+    return;
+  }
+#endif
   if (threadIdx.x == 0 && (first || last) && blockIdx.y == 0 && blockIdx.z == 0) {
     if (last) id += 16;
     unsigned long long t;

@@ -108,8 +108,11 @@ constexpr size_t att_smem_bytes() {
 // AttnParams::wo).  Warp w owns output features [w d / 8, (w + 1) d / 8); its weight fragments -- 16 rows x 64 columns
 // per group of rows, read with 16-byte loads whose eight elements are consecutive in K (the contraction index is
 // permuted identically for both MMA operands) -- are requested before the dependency wait, since weights never change.
-template <typename ActT, int DH, int QPW, bool FUSE = false>
-__global__ void __launch_bounds__(256)
+// MINB = 2 (at most 128 registers, two CTAs per SM) is for grids of more CTAs than SMs -- a batch of 8 rows x 4 query
+// chunks x 8 heads: measured, the second wave of such a 256-CTA grid doubled the kernel's time; grids that fit one wave
+// use MINB = 1, which keeps every CTA on an SM of its own.
+template <typename ActT, int DH, int QPW, bool FUSE = false, int MINB = 1>
+__global__ void __launch_bounds__(256, MINB)
 attention_kernel(const AttnParams p) {
   constexpr int R = DH / 32;                 // output dims per lane
   constexpr int QC = ATT_WARPS * QPW;        // queries per CTA
