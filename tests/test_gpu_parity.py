@@ -168,6 +168,46 @@ def test_mini_bf16_lockstep_and_generate():
     print(f"mini bf16 drafter at prefixes 3/11/0/17: {st}")
 
 
+def test_mini_bf16_long_targets_reach_the_key_parallel_attention():
+    """Targets of up to 300 tokens: self-attention rows hold hundreds of keys, so the verifier's block-causal attention
+    (per-token key counts) and the drafter's bidirectional attention over prefix + masks run in the kernel that spreads a
+    row's keys over the warps of a CTA (1, 2 and 4 query tiles per CTA; ragged rows of 270 and 130 committed tokens).
+    The verifier's block is compared with the checker's plain forward over the whole sequence (no cache)."""
+    shape = synth.MINI_BF16
+    dec, om, on = make(shape, 2, 20, 300, 20, drafter=True)
+    r = np.random.default_rng(31)
+    src = r.integers(4, shape.vocab, size=(2, 20)).astype(np.int32)
+    lens = np.array([20, 13], np.int32)
+    prefixes = [r.integers(4, shape.vocab, size=n).astype(np.int32) for n in (270, 130)]
+    st = P.drafter_at_prefix(dec, on, src, lens, prefixes, 20, TOL_BF16)
+    print(f"mini bf16 drafter at prefixes 270/130: {st}")
+    ks = [20, 9]
+    drafts = np.full((2, 20), -1, np.int32)
+    for b in range(2):
+        drafts[b, : ks[b]] = r.integers(4, shape.vocab, size=ks[b])
+    ids, n = dec.verify_block(drafts, ks)
+    lg = dec.debug_logits(sum(ks))
+    off, exact = 0, 0
+    for b in range(2):
+        k, j = ks[b], len(prefixes[b])
+        mem = om.encode_memory(src[b, : lens[b]])
+        seq = np.concatenate([[om.bos], prefixes[b], drafts[b, : k - 1]]).astype(np.int32)
+        ref = om.decode_full(mem, seq, causal=True)[j: j + k]
+        assert np.abs(lg[off: off + k] - ref).max() <= TOL_BF16
+        for i in range(k):
+            top = np.argsort(-ref[i], kind="stable")[:2]
+            if ref[i][top[0]] - ref[i][top[1]] > P.MARGIN:
+                assert ids[b, i] == top[0], (b, i)
+                exact += 1
+            else:
+                assert ids[b, i] in top
+        n_self, _ = P.OPS.accept(ids[b, :k], drafts[b, :k], eos=2)
+        assert n[b] == n_self
+        off += k
+    assert exact >= 5
+    dec.close()
+
+
 # ------------------------------------------------------------------------------------------ workloads 2, 3
 @pytest.fixture(scope="module")
 def base_weights():
