@@ -34,8 +34,13 @@ struct Mat {
 struct ActBuf {
   void* ptr = nullptr;
   int cols = 0;
-  CUtensorMap map[PK_COUNT];        // box rows = the pass's token tile
-  CUtensorMap map_half[PK_COUNT];   // box rows = half of it (used when the full tile would leave most SMs idle)
+  // one map per pass kind and token tile: box rows 16, 32, 64, 128, 256 (index log2(rows) - 4), up to the pass's own tile
+  CUtensorMap map[PK_COUNT][5];
+  const CUtensorMap& map_for(int pk, int tile) const {
+    int i = 0;
+    while ((16 << i) < tile && i < 4) ++i;
+    return map[pk][i];
+  }
 };
 struct EncLayer {
   Mat wqkv, wo, w1, w2;
@@ -68,7 +73,18 @@ struct PassCfg {
   // token dimension alone gives only a handful of tiles (power of two, divides the K blocks, <= max_split).
   // Token tile for a projection with N output features: the pass's tile, or half of a 256-token tile when the
   // full tile would give fewer CTAs than two per SM (the K loop costs the same per CTA either way).
+  // Token tile of a projection with N output features.  Up to 64 tokens: one tile (more, smaller tiles were measured
+  // slower for a 40-token block).  Beyond that the pass's kernels are latency-bound and smaller tiles win -- more CTAs,
+  // more MMA issuers per CTA, a shorter epilogue each -- until the grids outgrow the SMs; measured per step (base model):
+  //   100 / 120 / 128 tokens: 64-token tiles 277 / 289 / 293 us against 305 / 316 / 321 us with one 128-token tile;
+  //   200 / 240 tokens: 32-token tiles 331 / 305 us, 64: 344 / 311, 128: 364 / 336, 16: 372;
+  //   320 / 400 / 512 tokens: 64-token tiles 366 / 357 / 389 us against 415 / 410 / 458 (128) and 383 / 380 / 410 (32);
+  //   800 / 1024 tokens: 64-token tiles 455 / 468 us against 477 / 486 (128);  2048 tokens: 128-token tiles 543 us, 64: 571.
   int tile_for(int N, int n_sms) const {
+    if (M_cap <= 64) return ntile;
+    if (M_cap <= 128) return 64;
+    if (M_cap <= 256) return 32;
+    if (M_cap <= 1024) return 64;
     if (ntile == 256 && ((N + 127) / 128) * ((M_cap + 255) / 256) < 2 * n_sms) return 128;
     return ntile;
   }
@@ -527,7 +543,7 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
   }
   if (h->bf16) {
     p.ntile = h->pass[pk].tile_for(W.N, num_sms());
-    const CUtensorMap& mx = (p.ntile == h->pass[pk].ntile) ? X.map[pk] : X.map_half[pk];
+    const CUtensorMap& mx = X.map_for(pk, p.ntile);
     if (epi != EPI_F32) p.ksplit = 1;
     switch (epi) {
       case EPI_F32: e = launch_tc<EPI_F32>(h->stream, W.map, mx, p, M_cap); break;
@@ -536,7 +552,7 @@ int gemm(ad_handle* h, int epi, const Mat& W, const ActBuf& X, int pk, const int
       default:
         // (a pass with a 256-token tile also has the 128-row map of its token operand)
         e = (h->pass[pk].ntile == 256 && vocab_goes_persistent(W.K, W.N, M_cap, p.bias))
-                ? launch_vocab_persistent(h->stream, W.map, X.map_half[pk], p, M_cap)
+                ? launch_vocab_persistent(h->stream, W.map, X.map_for(pk, tc::P_TOK), p, M_cap)
                 : launch_tc<EPI_ARGMAX>(h->stream, W.map, mx, p, M_cap);
         break;
     }
@@ -1124,17 +1140,15 @@ extern "C" int ad_create(const ad_model_cfg* cfg, const ad_weights* w, void* wor
     bool ok = true;
     ActBuf* bufs[4] = {&h->yb, &h->abuf, &h->hbuf, &h->xg};
     for (ActBuf* b : bufs)
-      for (int k = 0; k < PK_COUNT; ++k) {
-        ok = ok && make_map(&b->map[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile);
-        ok = ok && make_map(&b->map_half[k], b->ptr, h->M_all, b->cols, h->pass[k].ntile / 2);
-      }
+      for (int k = 0; k < PK_COUNT; ++k)
+        for (int i = 0; i < 5 && (16 << i) <= h->pass[k].ntile; ++i)
+          ok = ok && make_map(&b->map[k][i], b->ptr, h->M_all, b->cols, 16 << i);
     if (cfg->has_drafter) {
       const int Me = h->pass[PK_ENCODE].M_cap, nt = h->pass[PK_ENCODE].ntile;
       ActBuf* sbufs[3] = {&h->side.yb, &h->side.abuf, &h->side.hbuf};
-      for (ActBuf* b : sbufs) {
-        ok = ok && make_map(&b->map[PK_ENCODE], b->ptr, Me, b->cols, nt);
-        ok = ok && make_map(&b->map_half[PK_ENCODE], b->ptr, Me, b->cols, nt / 2);
-      }
+      for (ActBuf* b : sbufs)
+        for (int i = 0; i < 5 && (16 << i) <= nt; ++i)
+          ok = ok && make_map(&b->map[PK_ENCODE][i], b->ptr, Me, b->cols, 16 << i);
     }
     if (!ok) return bail(AD_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   }
