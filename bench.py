@@ -80,8 +80,8 @@ def reduce_max_sum(dist, dev, seconds_or_ms, count):
 # DRAM counters of one verification step (dram__bytes_read.sum + dram__bytes_write.sum summed over the step's
 # kernels, ncu, caches flushed before every kernel) with the digest of the kernel sources they were taken on:
 # the figures are reported only while the sources still have that digest.
-NCU_COUNTERS = dict(sources_sha256="1e9604f567860b521cded6ea535eb106b63e47a30fc2c1dcd023ae6359e683c1",
-                    step_block40_bytes=102919168, projection_bytes=32862000,
+NCU_COUNTERS = dict(sources_sha256="37b384c806630e2500ef6aaa4768c3d2f2ff7fbb4bbcd742b10a556ea727aad6",
+                    step_block40_bytes=102930688, projection_bytes=32880640,
                     summary="profiles/verify_step_base_b1_k40_dram_traffic.txt")
 
 
