@@ -478,7 +478,10 @@ int tc_stages(int ntile, int kb, int n_ctas) {
   const int stage = tc::A_STAGE_BYTES + ntile * tc::BLOCK_K * 2;
   const int budget = n_ctas > num_sms() ? 100 * 1024 : 200 * 1024;
   int s = clampi(budget / stage, 1, tc::MAX_STAGES);
-  return s < kb ? s : (kb > 0 ? kb : 1);
+  if (s >= kb) return kb > 0 ? kb : 1;
+  // several ring rounds: the kernel's producer count divides the depth, so avoid the prime depths 5 and 7
+  if (s == 5 || s == 7) --s;
+  return s;
 }
 
 template <int EPI>

@@ -349,7 +349,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
   // TMA issue is spread over lane 0 of all eight warps: one thread's bulk-tensor copies are processed one after
   // the other, several threads' copies run side by side.  Stage i of the first ring round belongs to warp i;
-  // later rounds are fed by warps 0, 2 and 3.
+  // later rounds are fed by up to four of the warps 0 .. 3.
   if (early && lane == 0) {
     // weights never change: fetch the first ring round before the previous kernel has finished
     for (int i = warp; i < first_round; i += THREADS / 32) {
@@ -383,12 +383,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         did_s[j] = (t0 + j < M) ? p.draft_id[t0 + j] : -1;
       }
     }
-    if (lane == 0 && warp != 1 && warp < 4) {
+    if (lane == 0 && warp < 4) {
       // ---- TMA producers: everything that was not issued above ----
-      // No more producers than stages: a producer's consecutive K blocks are then at most one ring round apart,
-      // so its parity wait on an "empty" barrier can never alias a phase two rounds back.
-      const int pw = warp == 0 ? 0 : warp - 1;          // 0, 1, 2
-      const int nprod = stages < 3 ? stages : 3;
+      // The producer count divides the ring depth, so producer pw refills the same stages (pw, pw + nprod, ...) round
+      // after round and every stage is refilled by one thread only.  Its parity wait on a stage's "empty" barrier is
+      // then always for the phase right after the one it waited for last time on that stage.  (With a count that does
+      // not divide the depth a producer comes back to a stage only every few rounds; arriving early it would find the
+      // barrier an even number of phases behind, take the stale parity for the one it waits for, overwrite a stage
+      // that has not been consumed and arm its "full" barrier twice in one phase -- seen as an "unspecified launch
+      // failure" with 4 stages, 3 producers and 4 ring rounds.)
+      const int pw = warp;
+      int nprod = 1;
+      for (int cand = 4; cand > 1; --cand)
+        if (stages % cand == 0) { nprod = cand; break; }
       const int begin = early ? first_round : 0;
       for (int i = begin + pw; pw < nprod && i < num_kb; i += nprod) {
         const int s = i % stages;

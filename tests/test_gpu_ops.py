@@ -34,7 +34,11 @@ def test_fp32_linear(M, K, N):
 
 @pytest.mark.parametrize("M,K,N", [(1, 64, 128), (16, 64, 128), (64, 512, 1536), (25, 1024, 300), (200, 512, 512),
                                    (256, 2048, 640), (7, 4096, 128), (100, 2048, 384), (100, 192, 256),
-                                   (12, 320, 20000)])
+                                   (12, 320, 20000),
+                                   # K loops of several ring rounds with more CTAs than SMs (short rings): 4 stages x 4
+                                   # rounds and x 6 rounds with four issuers, a depth that would be 5 without the
+                                   # divisibility rule, 8 stages x 8 rounds
+                                   (64, 1024, 19200), (40, 1536, 19200), (16, 2048, 19200), (64, 4096, 256)])
 def test_bf16_tensor_core_linear(M, K, N):
     """Inputs are BF16-exact, the accumulator is FP32: only the summation order differs from the checker.
     The shapes walk through the kernel's configurations: one, two and four MMA issuers, K loops of one and of

@@ -291,6 +291,23 @@ def test_workload4_big_generalized():
     P.check_free_run(outs[0], greedy[0][0], greedy[0][1], "big")
 
 
+def test_big_model_batch_of_four():
+    """Transformer-big, four rows, 32-token sources, blocks of 25: passes of 100 and 128 tokens, whose projections run
+    K loops of several ring rounds (K = 1024 and 4096) on short rings shared by two CTAs per SM.  Rows 0 and 3 follow the
+    checker for two iterations; the other rows share their passes."""
+    shape = synth.BIG
+    dec, om, _ = make(shape, 4, 32, 50, 25)
+    r = np.random.default_rng(44)
+    src = r.integers(4, shape.vocab, size=(4, 32)).astype(np.int32)
+    lens = np.array([32, 20, 27, 32], np.int32)
+    max_len = np.full(4, 50, np.int32)
+    streams = [r.integers(4, shape.vocab, size=50).astype(np.int32) for _ in range(4)]
+    tot = P.lockstep(dec, om, src, lens, streams, 25, max_len, TOL_BF16, max_steps=2, check_rows=[0, 3])
+    print(f"big, batch 4, two iterations, rows 0 and 3: {tot}")
+    assert tot["steps"] == 2
+    dec.close()
+
+
 def test_workload5_base_long_source_batch8(base_weights):
     wl = synth.WORKLOADS[5]
     wn = synth.make_weights(synth.BASE, 1)
