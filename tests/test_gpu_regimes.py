@@ -1,0 +1,53 @@
+"""A property that holds at any size: a row's verified block does not depend on which other rows share its pass.
+
+Batched passes of different sizes take different kernels and launch shapes (token tiles of 32, 64 or 128, split-K
+factors, the attention kernel for few queries / many queries / hundreds of keys, the persistent projection kernel), a
+single row takes the small-pass ones.  The scores of sampled rows of a ragged batch are compared with the same rows
+verified alone; both sides are the library, so this pins no arithmetic -- the checker does that at sizes it can afford
+(test_gpu_parity.py) -- but it ties every large-pass configuration to the small-pass path the checker follows
+element by element.  Tolerance: the BF16 bar (the two sides differ in summation order only)."""
+import numpy as np
+import pytest
+
+from paper_2205_10350_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+CASES = [("base", synth.BASE, 8, 25, 400),       # 200-token capacity: 32-token tiles, keys spread over warps
+         ("base", synth.BASE, 32, 30, 48),       # 960: 64-token tiles, tensor-core attention, persistent projection
+         ("big", synth.BIG, 4, 25, 32),          # 100: K loops of several ring rounds
+         ("big", synth.BIG, 16, 64, 32),         # 1024
+         ("bart", synth.BART_BASE_SIZED, 6, 30, 40),   # 12 heads, K blocks not a power of two
+         ("base", synth.BASE, 3, 64, 300)]       # 192: long sources with long blocks
+
+
+@pytest.mark.parametrize("name,shape,B,k,S", CASES, ids=[f"{c[0]}-{c[2]}x{c[3]}-src{c[4]}" for c in CASES])
+def test_batched_pass_agrees_with_single_row_passes(name, shape, B, k, S):
+    r = np.random.default_rng(B * 1000 + k)
+    w = synth.make_weights(shape, 0)
+    src = r.integers(4, shape.vocab, size=(B, S)).astype(np.int32)
+    lens = r.integers(max(1, S // 2), S + 1, size=B).astype(np.int32)
+    ks = r.integers(1, k + 1, size=B).astype(np.int32)
+    ks[B - 1] = k                                         # one full-length block
+    drafts = r.integers(4, shape.vocab, size=(B, k)).astype(np.int32)
+    dec = binding.AggressiveDecoder(shape, w, max_batch=B, max_src=S, max_tgt=k, kmax=k)
+    dec.encode(src, lens)
+    ids, n = dec.verify_block(drafts, ks)
+    lg = dec.debug_logits(int(ks.sum()))
+    dec.close()
+    offs = np.concatenate([[0], np.cumsum(ks)])
+    one = binding.AggressiveDecoder(shape, w, max_batch=1, max_src=S, max_tgt=k, kmax=k)
+    worst = 0.0
+    for b in sorted({0, B // 2, B - 1}):
+        one.encode(src[b: b + 1], lens[b: b + 1])
+        ids1, n1 = one.verify_block(drafts[b: b + 1], ks[b: b + 1])
+        l1 = one.debug_logits(int(ks[b]))
+        got = lg[offs[b]: offs[b + 1]]
+        worst = max(worst, float(np.abs(got - l1).max()))
+        # ids agree wherever the single-row scores leave no doubt
+        top2 = np.sort(l1, axis=1)[:, -2:]
+        clear = (top2[:, 1] - top2[:, 0]) > 0.1
+        assert (ids[b, : ks[b]][clear] == ids1[0, : ks[b]][clear]).all()
+    one.close()
+    print(f"{name} B={B} k={k} S={S}: worst |batched - alone| = {worst:.4f}")
+    assert worst <= 5e-2
