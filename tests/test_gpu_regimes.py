@@ -51,3 +51,47 @@ def test_batched_pass_agrees_with_single_row_passes(name, shape, B, k, S):
     one.close()
     print(f"{name} B={B} k={k} S={S}: worst |batched - alone| = {worst:.4f}")
     assert worst <= 5e-2
+
+
+DRAFT_CASES = [("base", synth.BASE, 8, 25, 400, 40), ("big", synth.BIG, 4, 25, 40, 30), ("mini", synth.MINI_BF16, 6, 16, 30, 200)]
+
+
+@pytest.mark.parametrize("name,shape,B,k,S,T", DRAFT_CASES, ids=[f"{c[0]}-{c[2]}rows-prefix<={c[5]}" for c in DRAFT_CASES])
+def test_batched_drafter_pass_agrees_with_single_row_passes(name, shape, B, k, S, T):
+    """The same for the drafter's pass (Section 3.2.1): rows are walked to ragged prefixes by teacher forcing, then the
+    draft scores of sampled rows of the batch are compared with the same rows drafted alone."""
+    r = np.random.default_rng(B * 100 + T)
+    w, wn = synth.make_weights(shape, 0), synth.make_weights(shape, 1)
+    src = r.integers(4, shape.vocab, size=(B, S)).astype(np.int32)
+    lens = r.integers(max(1, S // 2), S + 1, size=B).astype(np.int32)
+    prefixes = [r.integers(4, shape.vocab, size=int(n)).astype(np.int32) for n in r.integers(0, T + 1, size=B)]
+
+    def draft(dec, rows):
+        dec.encode(src[rows], lens[rows])
+        done = [0] * len(rows)
+        while any(done[i] < len(prefixes[b]) for i, b in enumerate(rows)):
+            ks = np.zeros(len(rows), np.int32)
+            toks = np.full((len(rows), dec.kmax), -1, np.int32)
+            for i, b in enumerate(rows):
+                seg = prefixes[b][done[i]: done[i] + dec.kmax]
+                ks[i] = len(seg)
+                toks[i, : len(seg)] = seg
+                done[i] += len(seg)
+            dec.verify_block(toks, ks)
+            dec.force_commit(toks, ks)
+        d, kk = dec.draft_block(k)
+        return d, kk, dec.debug_logits(int(kk.sum()), which=1)
+
+    dec = binding.AggressiveDecoder(shape, w, wn, max_batch=B, max_src=S, max_tgt=T + k, kmax=k)
+    d, kk, scores = draft(dec, list(range(B)))
+    dec.close()
+    offs = np.concatenate([[0], np.cumsum(kk)])
+    one = binding.AggressiveDecoder(shape, w, wn, max_batch=1, max_src=S, max_tgt=T + k, kmax=k)
+    worst = 0.0
+    for b in sorted({0, B // 2, B - 1}):
+        d1, k1, s1 = draft(one, [b])
+        assert int(k1[0]) == int(kk[b])
+        worst = max(worst, float(np.abs(scores[offs[b]: offs[b + 1]] - s1).max()))
+    one.close()
+    print(f"{name} B={B}: drafter worst |batched - alone| = {worst:.4f}")
+    assert worst <= 5e-2
