@@ -80,8 +80,8 @@ def reduce_max_sum(dist, dev, seconds_or_ms, count):
 # DRAM counters of one verification step (dram__bytes_read.sum + dram__bytes_write.sum summed over the step's
 # kernels, ncu, caches flushed before every kernel) with the digest of the kernel sources they were taken on:
 # the figures are reported only while the sources still have that digest.
-NCU_COUNTERS = dict(sources_sha256="37b384c806630e2500ef6aaa4768c3d2f2ff7fbb4bbcd742b10a556ea727aad6",
-                    step_block40_bytes=102930688, projection_bytes=32880640,
+NCU_COUNTERS = dict(sources_sha256="ef1170edd47f7cb51e5fa18cdb5a8348d5a0885c56b78a4d3f46eafb7ea5cda6",
+                    step_block40_bytes=102913536, projection_bytes=32859392,
                     summary="profiles/verify_step_base_b1_k40_dram_traffic.txt")
 
 
