@@ -95,3 +95,43 @@ def test_batched_drafter_pass_agrees_with_single_row_passes(name, shape, B, k, S
     one.close()
     print(f"{name} B={B}: drafter worst |batched - alone| = {worst:.4f}")
     assert worst <= 5e-2
+
+
+LOOP_CASES = [(5, 64, 40, "IAD", False), (8, 25, 100, "GAD", True), (32, 64, 48, "IAD", False), (4, 40, 300, "GAD", True)]
+
+
+@pytest.mark.parametrize("B,k,S,mode,drafter", LOOP_CASES, ids=[f"{c[3]}-{c[0]}rows-k{c[1]}-src{c[2]}" for c in LOOP_CASES])
+def test_decode_loop_as_one_graph_equals_direct_launches_at_every_pass_size(B, k, S, mode, drafter):
+    """The whole loop (Algorithm 1 / Section 3.2) on the base model at several batch sizes: one graph launch with the
+    device-side loop, the same call again, and direct launches with host polling must return identical tokens and
+    iteration counts.  How many rows also equal the library's own greedy decoding (block size 1, other kernels and launch
+    shapes) is printed: the method is lossless, so every row whose positions are all clear of near-ties does."""
+    shape = synth.BASE
+    r = np.random.default_rng(B * 7 + k)
+    w = synth.make_weights(shape, 0)
+    wn = synth.make_weights(shape, 1) if drafter else None
+    T = max(48, k)
+    dec = binding.AggressiveDecoder(shape, w, wn, max_batch=B, max_src=S, max_tgt=T, kmax=k)
+    src = r.integers(4, shape.vocab, size=(B, S)).astype(np.int32)
+    lens = r.integers(max(1, S // 2), S + 1, size=B).astype(np.int32)
+    max_len = r.integers(8, T + 1, size=B).astype(np.int32)
+    g, _ = dec.generate(src, lens, mode="IAD", k=1, max_len=max_len)
+    gg = np.full((B, T), synth.PAD, np.int32)
+    for b in range(B):
+        gg[b, : len(g[b])] = g[b]
+    kw = dict(mode=mode, k=k, max_len=max_len)
+    if drafter:
+        kw["run_drafter"] = True
+    else:
+        kw["draft_override"] = synth.corrupt_stream(gg, [len(x) for x in g], 0.8, shape.vocab, 3, B)
+    a, sa = dec.generate(src, lens, use_graph=True, **kw)
+    d, sd = dec.generate(src, lens, use_graph=False, **kw)
+    c, sc = dec.generate(src, lens, use_graph=True, **kw)
+    for b in range(B):
+        assert np.array_equal(a[b], d[b]) and np.array_equal(a[b], c[b]), b
+        assert 1 <= len(a[b]) <= max_len[b]
+    assert sa["iterations"] == sd["iterations"] == sc["iterations"]
+    same = sum(np.array_equal(a[b], g[b]) for b in range(B))
+    print(f"B={B} k={k} S={S} {mode}: {sa['iterations']} iterations, {same}/{B} rows identical to block-size-1 decoding")
+    assert same >= B - max(1, B // 4)          # near-ties may move a few rows off; a broken loop moves all of them
+    dec.close()
