@@ -92,10 +92,12 @@ struct PassCfg {
     const int tiles = ((N + 127) / 128) * ((M_cap + tile - 1) / tile);
     const int kb = K / 64;
     int s = 1;
-    // Few tokens (one or two token tiles): at most ~3/4 of the SMs.  Measured, a 128-CTA split-K grid of these
-    // one-CTA-per-SM kernels ran 16 of its CTAs as a second wave behind the predecessor it overlaps (9.5 us instead of
-    // 5.3 us).  With many tokens the grid has several waves anyway and the split keeps the K loops short.
-    const int cap = M_cap <= 256 ? 112 : 160;
+    // Up to 256 tokens: at most one CTA per SM.  (With 128-token tiles a 128-CTA grid of these one-CTA-per-SM kernels ran
+    // 16 of its CTAs as a second wave behind the 32 CTAs of the projection before it; with the 32- and 64-token tiles such
+    // passes take now the projection before it fills the SMs itself and the full-width split is as fast or faster: big
+    // model, 100 tokens, 392 against 417 us per step.)  With many tokens the grid has several waves anyway and the split
+    // keeps the K loops short.
+    const int cap = M_cap <= 256 ? 148 : 160;
     while (s * 2 <= max_split && tiles * s * 2 <= cap && kb % (s * 2) == 0) s *= 2;
     return s;
   }
