@@ -97,7 +97,8 @@ struct PassCfg {
     // passes take now the projection before it fills the SMs itself and the full-width split is as fast or faster: big
     // model, 100 tokens, 392 against 417 us per step.)  With many tokens the grid has several waves anyway and the split
     // keeps the K loops short.
-    const int cap = M_cap <= 256 ? 148 : 160;
+    // (a single token tile, up to 64 tokens: 112 -- the big model's 25-token pass loses 4 % with 128 one-K-block CTAs)
+    const int cap = M_cap <= 64 ? 112 : (M_cap <= 256 ? 148 : 160);
     while (s * 2 <= max_split && tiles * s * 2 <= cap && kb % (s * 2) == 0) s *= 2;
     return s;
   }
