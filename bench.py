@@ -585,6 +585,21 @@ def bench_extras(args, binding, dec, w, dev, pk, flush, t_src, t_len, t_max, t_o
                                    frac_of_floor=flops32 / (pk["bf16_tflops"] * 1e12) * 1e6 / us32,
                                    frac_of_sustained=flops32 / (pk["bf16_tflops_sustained"] * 1e12) * 1e6 / us32,
                                    note="batch 32, block 64, empty prefix, source 64; direct launches, weights L2-warm")
+    # the one kernel of that step with tensor-core-sized work, timed alone: projection + arg-max partials over 2048 tokens
+    x32 = torch.randn((M32, d), device=dev).bfloat16()
+    nb32 = lib.ad_vocab_argmax_scratch_bytes(V, M32)
+    scratch32 = torch.empty(nb32 + 256, dtype=torch.uint8, device=dev)
+    sbase32 = (scratch32.data_ptr() + 255) // 256 * 256
+
+    def vocab32_once():
+        assert lib.ad_vocab_argmax(C.c_void_p(x32.data_ptr()), C.c_void_p(emb.data_ptr()), 1, M32, d, V, None, C.c_void_p(sbase32), nb32,
+                                   C.c_void_p(status.data_ptr()), C.c_void_p(dec.stream.cuda_stream)) == 0
+    t_v32 = statistics.mean(_events(dec.stream, vocab32_once, 20))
+    fl_v32 = 2.0 * M32 * V * d
+    extras["tensor_regime"]["projection_kernel"] = dict(
+        kernel="vocab_argmax_persistent_kernel, vocabulary 32000 x 512, 2048 tokens", us=t_v32, flops=fl_v32,
+        tflops=fl_v32 / (t_v32 * 1e-6) / 1e12, frac_of_burst_peak=fl_v32 / (t_v32 * 1e-6) / 1e12 / pk["bf16_tflops"],
+        note="timed alone with CUDA events (weights L2-warm); ncu counters in profiles/vocab_argmax_persistent_base_M2048_ncu_full.txt")
 
     # the other workload recipes (and shapes) through ad_generate, the CPU checker's bounded sample beside each
     if not args.skip_workloads:
