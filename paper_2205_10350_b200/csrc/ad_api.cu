@@ -695,7 +695,9 @@ int layernorm(ad_handle* h, const PassCfg& pc, int nsplit, const float* bias, co
                               (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
     else e = launch_k(layernorm_rows_kernel<float>, rgrid, dim3(256), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                       (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
-  } else if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
+  } else if (h->bf16 && d > 512) e = launch_k(layernorm_kernel<bf16, 256>, grid, dim3(256), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
+                            (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
+  else if (h->bf16) e = launch_k(layernorm_kernel<bf16>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                             (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (bf16*)h->yb.ptr);
   else e = launch_k(layernorm_kernel<float>, grid, dim3(128), 0, h->stream, (const int*)pc.plan.M, pre_src, nsplit, stride, bias,
                     (const float*)h->y, g, b, d, h->cfg.ln_eps, h->y, (float*)h->yb.ptr);
