@@ -80,8 +80,8 @@ def reduce_max_sum(dist, dev, seconds_or_ms, count):
 # DRAM counters of one verification step (dram__bytes_read.sum + dram__bytes_write.sum summed over the step's
 # kernels, ncu, caches flushed before every kernel) with the digest of the kernel sources they were taken on:
 # the figures are reported only while the sources still have that digest.
-NCU_COUNTERS = dict(sources_sha256="96338845390a2ecdff4f015f3601423f55158a39c5d1629c0482ed4fb98e6c75",
-                    step_block40_bytes=102919936, projection_bytes=32858112,
+NCU_COUNTERS = dict(sources_sha256="748bbf674820a70485669346e6d0b8a7256ee158b313d80ee57d22edeb6d6edc",
+                    step_block40_bytes=102923008, projection_bytes=32858368,
                     summary="profiles/verify_step_base_b1_k40_dram_traffic.txt")
 
 
